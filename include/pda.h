@@ -1,0 +1,178 @@
+/* pda.h -- C ABI of the B200 (sm_100a) paged decode attention library (libpda.so).
+ *
+ * One decode step of one attention layer over a paged KV cache:
+ *
+ *     kv_append  ->  paged_decode_attention  ( ->  paged_decode_reduce )
+ *
+ * The operation is the one the serving stacks of the paper run at every decode
+ * step on top of their "paged KV cache" with grouped-query attention ("32 query
+ * heads sharing 8 key/value heads", Appendix A, Scenario A): for sequence b and
+ * query head h, with kv head g = h / (num_q_heads / num_kv_heads),
+ *
+ *     out[b,h,:] = softmax_j( scale * q[b,h,:] . K_j[g,:] ) . V_j[g,:]
+ *
+ * over the sequence's tokens j = 0 .. seq_lens[b]-1 in logical order, token j
+ * living in physical page block_table[b][j / page_size], slot j % page_size.
+ * The paper names these ingredients but defines no layout; everything below is
+ * this library's definition.
+ *
+ * Conventions
+ *   - All data pointers are DEVICE pointers unless a comment says "host".
+ *   - The caller owns every buffer. The library allocates no device memory and
+ *     keeps no device state between calls (it memoises TMA descriptors on the
+ *     host, keyed by pointer and shape).
+ *   - Every call enqueues work on `stream` (a cudaStream_t passed as void*) and
+ *     returns without synchronising. Nothing reads seq_lens or block_table back
+ *     to the host, so a step can be captured in a CUDA graph.
+ *   - Return value: 0 = PDA_OK; < 0 = PDA_ERR_* detected on the host before
+ *     anything was enqueued; > 0 = the cudaError_t of a failed launch.
+ *   - `status` (optional, device int32, caller-zeroed): problems found on the
+ *     device are recorded with atomicMax(status, PDA_DEV_*). The affected unit's
+ *     output is zero-filled; no out-of-bounds access is ever made.
+ *   - bf16 = upper half of an IEEE binary32. e4m3 = OCP FP8 E4M3 (bias 7, max
+ *     finite 448, no infinities, S.1111.111 = NaN).
+ */
+#ifndef PDA_H_
+#define PDA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PDA_VERSION 100
+
+/* host-side return codes */
+#define PDA_OK 0
+#define PDA_ERR_INVALID_ARG (-1)  /* null pointer, negative size, inconsistent sizes          */
+#define PDA_ERR_UNSUPPORTED (-2)  /* shape / dtype / stride outside the supported set          */
+#define PDA_ERR_MISALIGNED (-3)   /* a pointer or stride breaks the 16-byte alignment rule     */
+#define PDA_ERR_TOO_LARGE (-4)    /* size beyond a documented fixed maximum                    */
+
+/* device-side status codes (atomicMax into *status) */
+#define PDA_DEV_OK 0
+#define PDA_DEV_BAD_PAGE 1     /* block_table entry outside [0, num_pages) for a live page     */
+#define PDA_DEV_BAD_SEQ_LEN 2  /* seq_lens[b] > block_table_stride * page_size                 */
+#define PDA_DEV_TIMEOUT 3      /* a bounded wait on an asynchronous copy expired               */
+
+/* KV element types */
+#define PDA_BF16 0
+#define PDA_FP8_E4M3 1
+
+/* flags for paged_decode_attention */
+#define PDA_FLAG_FORCE_GENERIC 1u /* use the plain CUDA-core kernel even where the
+                                     TMA + tensor-core kernel applies (for testing) */
+
+typedef void* pda_stream_t; /* cudaStream_t */
+
+/* Describes k_cache and v_cache (both have the same geometry).
+ * Element (page, head, slot, d) lives at element offset
+ *   page*page_stride + head*head_stride + slot*slot_stride + d.
+ * The canonical layout is [num_pages, num_kv_heads, page_size, head_dim]
+ * contiguous, i.e. slot_stride = head_dim, head_stride = page_size*head_dim,
+ * page_stride = num_kv_heads*head_stride; any strides whose byte values are
+ * multiples of 16 are accepted. */
+typedef struct pda_cache_desc {
+  int64_t page_stride;  /* elements */
+  int64_t head_stride;  /* elements */
+  int64_t slot_stride;  /* elements */
+  int32_t num_pages;
+  int32_t page_size;    /* tokens per page; supported: 16 */
+  int32_t num_kv_heads;
+  int32_t head_dim;     /* supported: multiples of 32 up to 256; fast path 64 and 128 */
+  int32_t dtype;        /* PDA_BF16 or PDA_FP8_E4M3 */
+} pda_cache_desc;
+
+int pda_version(void);
+const char* pda_status_string(int code); /* text for a PDA_ERR_* / PDA_DEV_* / 0 code */
+
+/* ceil(max_seq_len / chunk_tokens): the `max_chunks` extent the partial buffers need. */
+int pda_max_chunks(int32_t max_seq_len, int32_t chunk_tokens);
+
+/* KV append (this step's scatter of new keys/values into the paged cache; the
+ * paper's Appendix A lists the paged KV cache, not its update rule -- this is
+ * the plain definition): for every sequence b with L = seq_lens[b] > 0 (length
+ * AFTER the append) and every kv head g,
+ *     cache[block_table[b][(L-1)/P]][g][(L-1)%P][:] = new[b][g][:]   (bytewise)
+ * k_new, v_new: [batch, num_kv_heads, head_dim] bf16, contiguous. bf16 caches
+ * only (PDA_ERR_UNSUPPORTED for e4m3). Target slots must be distinct across the
+ * batch. A bad page id or length skips that sequence and sets *status.
+ * desc is a host pointer, read during the call. */
+int kv_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+              const pda_cache_desc* desc, const int32_t* block_table,
+              int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+              int32_t* status, pda_stream_t stream);
+
+/* Paged decode attention (definition at the top of this file; GQA head grouping
+ * per Appendix A, Scenario A).
+ *   q            [batch, num_q_heads, head_dim] bf16, contiguous
+ *   k_scale,
+ *   v_scale      [num_pages, num_kv_heads] fp32 dequantisation factors for e4m3
+ *                caches (value = decode(byte) * scale); NULL for bf16 caches
+ *   block_table  [batch, block_table_stride] int32; entries at or beyond
+ *                ceil(seq_lens[b]/page_size) are never read
+ *   scale        fp32 multiplier of q.k
+ *   chunk_tokens 0: whole sequence per unit, result written to `out`
+ *                [batch, num_q_heads, head_dim] bf16 (round to nearest even);
+ *                a sequence of length 0 gives zeros.
+ *                >0 (multiple of page_size): split-KV. Chunk c covers tokens
+ *                [c*chunk_tokens, min((c+1)*chunk_tokens, L)); for every c <
+ *                ceil(L/chunk_tokens) the kernel writes
+ *                  part_o  [batch, num_q_heads, max_chunks, head_dim] fp32,
+ *                          normalised within the chunk, and
+ *                  part_lse[batch, num_q_heads, max_chunks] fp32 = m + ln(l)
+ *                          (natural log of the chunk's softmax denominator);
+ *                other entries are left untouched; `out` is not written.
+ *                max_chunks * chunk_tokens must cover block_table_stride*page_size
+ *                or at least every seq_lens[b] (longer sequences set *status).
+ *   flags        PDA_FLAG_* bits
+ * Unused slots of a last page, unused pages and table tails may hold any bit
+ * pattern (NaN included). e4m3 caches: q is converted to fp16 for the tensor
+ * core path, so |q| must stay below 65504.
+ * Supported: page_size 16; num_q_heads a multiple of num_kv_heads; any group
+ * size and head_dim (multiple of 32, <= 256) on the generic kernel; group size
+ * <= 8 with head_dim 64 or 128 on the TMA + tensor-core kernel. */
+int paged_decode_attention(const void* q, const void* k_cache, const void* v_cache,
+                           const pda_cache_desc* desc, const float* k_scale,
+                           const float* v_scale, const int32_t* block_table,
+                           int32_t block_table_stride, const int32_t* seq_lens,
+                           int32_t batch, int32_t num_q_heads, float scale,
+                           int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                           int32_t max_chunks, uint32_t flags, int32_t* status,
+                           pda_stream_t stream);
+
+/* Merge of split-KV partials (the reduce step of flash-decoding; exact algebra):
+ *     out[b,h,:] = sum_c w_c part_o[b,h,c,:] / sum_c w_c,
+ *     w_c = exp(part_lse[b,h,c] - max_c part_lse[b,h,c]),  c < ceil(L_b/chunk_tokens)
+ * out: [batch, num_q_heads, head_dim] bf16. A sequence without chunks gives zeros. */
+int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
+                        int32_t batch, int32_t num_q_heads, int32_t head_dim,
+                        int32_t chunk_tokens, int32_t max_chunks, void* out,
+                        pda_stream_t stream);
+
+/* One whole decode step driven from HOST buffers (the end-to-end call): copies
+ * this step's q, k_new, v_new, seq_lens and block_table from (ideally pinned)
+ * host memory into the caller's device staging buffers, runs kv_append,
+ * paged_decode_attention and (chunk_tokens > 0) paged_decode_reduce, and copies
+ * `out` back to out_host; all on `stream`, without synchronising. The KV cache
+ * itself stays resident on the device between steps. *_dev are device buffers
+ * of the same sizes as their host counterparts. */
+int paged_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,
+                           const int32_t* block_table_host, const int32_t* seq_lens_host,
+                           void* q_dev, void* k_new_dev, void* v_new_dev,
+                           int32_t* block_table_dev, int32_t* seq_lens_dev,
+                           void* k_cache, void* v_cache, const pda_cache_desc* desc,
+                           int32_t block_table_stride, int32_t batch, int32_t num_q_heads,
+                           float scale, int32_t chunk_tokens, float* part_o, float* part_lse,
+                           int32_t max_chunks, void* out_dev, void* out_host, int32_t* status,
+                           pda_stream_t stream);
+
+/* Diagnostic: decodes all 256 e4m3 bytes with the device decoder the generic
+ * kernel uses; out256: device float[256]. */
+int pda_debug_e4m3_decode(float* out256, pda_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PDA_H_ */

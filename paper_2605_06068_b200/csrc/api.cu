@@ -1,0 +1,222 @@
+// C ABI of libpda: argument validation on the host, then kernel dispatch.
+#include <cstdint>
+
+#include "common.cuh"
+
+namespace {
+
+using pda::AttnParams;
+using pda::CacheGeom;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks the cache descriptor; on success fills `g`.
+int check_desc(const pda_cache_desc* d, CacheGeom* g) {
+  if (d == nullptr) return PDA_ERR_INVALID_ARG;
+  if (d->num_pages < 0 || d->num_kv_heads <= 0 || d->head_dim <= 0 || d->page_size <= 0)
+    return PDA_ERR_INVALID_ARG;
+  if (d->dtype != PDA_BF16 && d->dtype != PDA_FP8_E4M3) return PDA_ERR_UNSUPPORTED;
+  if (d->page_size != pda::kPageSize) return PDA_ERR_UNSUPPORTED;
+  if (d->head_dim % 32 != 0 || d->head_dim > 256) return PDA_ERR_UNSUPPORTED;
+  if (d->page_stride <= 0 || d->head_stride <= 0 || d->slot_stride < d->head_dim)
+    return PDA_ERR_INVALID_ARG;
+  const int64_t eb = d->dtype == PDA_BF16 ? 2 : 1;
+  if ((d->page_stride * eb) % 16 || (d->head_stride * eb) % 16 || (d->slot_stride * eb) % 16)
+    return PDA_ERR_MISALIGNED;
+  g->page_stride = d->page_stride;
+  g->head_stride = d->head_stride;
+  g->slot_stride = d->slot_stride;
+  g->num_pages = d->num_pages;
+  g->num_kv_heads = d->num_kv_heads;
+  g->head_dim = d->head_dim;
+  g->dtype = d->dtype;
+  return PDA_OK;
+}
+
+int check_attention(const void* q, const void* k_cache, const void* v_cache,
+                    const pda_cache_desc* desc, const float* k_scale, const float* v_scale,
+                    const int32_t* block_table, int32_t block_table_stride,
+                    const int32_t* seq_lens, int32_t batch, int32_t num_q_heads,
+                    int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                    int32_t max_chunks, AttnParams* p) {
+  CacheGeom g;
+  if (int rc = check_desc(desc, &g)) return rc;
+  if (batch < 0 || num_q_heads <= 0 || block_table_stride < 0 || chunk_tokens < 0)
+    return PDA_ERR_INVALID_ARG;
+  if (num_q_heads % g.num_kv_heads != 0) return PDA_ERR_INVALID_ARG;
+  if (chunk_tokens % pda::kPageSize != 0) return PDA_ERR_INVALID_ARG;
+  if (batch > 65535 || num_q_heads > 65535) return PDA_ERR_TOO_LARGE;
+  if (batch > 0) {
+    if (!q || !k_cache || !v_cache || !block_table || !seq_lens) return PDA_ERR_INVALID_ARG;
+    if (block_table_stride == 0) return PDA_ERR_INVALID_ARG;
+    if (g.dtype == PDA_FP8_E4M3 && (!k_scale || !v_scale)) return PDA_ERR_INVALID_ARG;
+    if (chunk_tokens == 0) {
+      if (!out) return PDA_ERR_INVALID_ARG;
+    } else {
+      if (!part_o || !part_lse || max_chunks <= 0) return PDA_ERR_INVALID_ARG;
+    }
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) ||
+        (chunk_tokens == 0 && !aligned16(out)) || (chunk_tokens > 0 && !aligned16(part_o)))
+      return PDA_ERR_MISALIGNED;
+  }
+  p->q = static_cast<const __nv_bfloat16*>(q);
+  p->k_cache = k_cache;
+  p->v_cache = v_cache;
+  p->k_scale = k_scale;
+  p->v_scale = v_scale;
+  p->block_table = block_table;
+  p->seq_lens = seq_lens;
+  p->out = static_cast<__nv_bfloat16*>(out);
+  p->part_o = part_o;
+  p->part_lse = part_lse;
+  p->status = nullptr;
+  p->geom = g;
+  p->block_table_stride = block_table_stride;
+  p->batch = batch;
+  p->num_q_heads = num_q_heads;
+  p->group = num_q_heads / g.num_kv_heads;
+  p->chunk_tokens = chunk_tokens;
+  p->max_chunks = max_chunks;
+  p->scale = 0.f;
+  return PDA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pda_version(void) { return PDA_VERSION; }
+
+const char* pda_status_string(int code) {
+  switch (code) {
+    case PDA_OK: return "ok";
+    case PDA_ERR_INVALID_ARG: return "invalid argument";
+    case PDA_ERR_UNSUPPORTED: return "unsupported shape, dtype or layout";
+    case PDA_ERR_MISALIGNED: return "pointer or stride not 16-byte aligned";
+    case PDA_ERR_TOO_LARGE: return "size beyond a fixed maximum";
+    case PDA_DEV_BAD_PAGE: return "device: block_table entry out of range";
+    case PDA_DEV_BAD_SEQ_LEN: return "device: seq_len exceeds block_table capacity";
+    case PDA_DEV_TIMEOUT: return "device: bounded wait on an asynchronous copy expired";
+    default: return code > 0 ? "cuda error or unknown device status" : "unknown error";
+  }
+}
+
+int pda_max_chunks(int32_t max_seq_len, int32_t chunk_tokens) {
+  if (chunk_tokens <= 0 || max_seq_len < 0) return PDA_ERR_INVALID_ARG;
+  return static_cast<int>((static_cast<int64_t>(max_seq_len) + chunk_tokens - 1) / chunk_tokens);
+}
+
+int kv_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+              const pda_cache_desc* desc, const int32_t* block_table,
+              int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+              int32_t* status, pda_stream_t stream) {
+  CacheGeom g;
+  if (int rc = check_desc(desc, &g)) return rc;
+  if (g.dtype != PDA_BF16) return PDA_ERR_UNSUPPORTED;
+  if (batch < 0 || block_table_stride < 0) return PDA_ERR_INVALID_ARG;
+  if (batch == 0) return PDA_OK;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !seq_lens ||
+      block_table_stride == 0)
+    return PDA_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache))
+    return PDA_ERR_MISALIGNED;
+  return static_cast<int>(pda::launch_kv_append(k_new, v_new, k_cache, v_cache, g, block_table,
+                                                block_table_stride, seq_lens, batch, status,
+                                                static_cast<cudaStream_t>(stream)));
+}
+
+int paged_decode_attention(const void* q, const void* k_cache, const void* v_cache,
+                           const pda_cache_desc* desc, const float* k_scale,
+                           const float* v_scale, const int32_t* block_table,
+                           int32_t block_table_stride, const int32_t* seq_lens,
+                           int32_t batch, int32_t num_q_heads, float scale,
+                           int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                           int32_t max_chunks, uint32_t flags, int32_t* status,
+                           pda_stream_t stream) {
+  AttnParams p;
+  if (int rc = check_attention(q, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                               block_table_stride, seq_lens, batch, num_q_heads, chunk_tokens,
+                               out, part_o, part_lse, max_chunks, &p))
+    return rc;
+  if (batch == 0) return PDA_OK;
+  p.status = status;
+  p.scale = scale;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (!(flags & PDA_FLAG_FORCE_GENERIC) && pda::attention_tma_supports(p))
+    return static_cast<int>(pda::launch_attention_tma(p, s));
+  return static_cast<int>(pda::launch_attention_generic(p, s));
+}
+
+int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
+                        int32_t batch, int32_t num_q_heads, int32_t head_dim,
+                        int32_t chunk_tokens, int32_t max_chunks, void* out,
+                        pda_stream_t stream) {
+  if (batch < 0 || num_q_heads <= 0 || head_dim <= 0 || chunk_tokens <= 0 || max_chunks <= 0)
+    return PDA_ERR_INVALID_ARG;
+  if (batch > 65535 || num_q_heads > 65535) return PDA_ERR_TOO_LARGE;
+  if (batch == 0) return PDA_OK;
+  if (!part_o || !part_lse || !seq_lens || !out) return PDA_ERR_INVALID_ARG;
+  return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
+                                             head_dim, chunk_tokens, max_chunks,
+                                             static_cast<__nv_bfloat16*>(out),
+                                             static_cast<cudaStream_t>(stream)));
+}
+
+int paged_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,
+                           const int32_t* block_table_host, const int32_t* seq_lens_host,
+                           void* q_dev, void* k_new_dev, void* v_new_dev,
+                           int32_t* block_table_dev, int32_t* seq_lens_dev,
+                           void* k_cache, void* v_cache, const pda_cache_desc* desc,
+                           int32_t block_table_stride, int32_t batch, int32_t num_q_heads,
+                           float scale, int32_t chunk_tokens, float* part_o, float* part_lse,
+                           int32_t max_chunks, void* out_dev, void* out_host, int32_t* status,
+                           pda_stream_t stream) {
+  AttnParams p;
+  if (!out_dev || !out_host) return PDA_ERR_INVALID_ARG;
+  if (int rc = check_attention(q_dev, k_cache, v_cache, desc, nullptr, nullptr, block_table_dev,
+                               block_table_stride, seq_lens_dev, batch, num_q_heads,
+                               chunk_tokens, out_dev, part_o, part_lse, max_chunks, &p))
+    return rc;
+  if (p.geom.dtype != PDA_BF16) return PDA_ERR_UNSUPPORTED;
+  if (batch == 0) return PDA_OK;
+  if (!q_host || !k_new_host || !v_new_host || !block_table_host || !seq_lens_host ||
+      !k_new_dev || !v_new_dev)
+    return PDA_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t D = p.geom.head_dim;
+  const size_t q_bytes = static_cast<size_t>(batch) * num_q_heads * D * 2;
+  const size_t new_bytes = static_cast<size_t>(batch) * p.geom.num_kv_heads * D * 2;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, s))) return e;
+  if ((e = cudaMemcpyAsync(k_new_dev, k_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
+  if ((e = cudaMemcpyAsync(v_new_dev, v_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
+  if ((e = cudaMemcpyAsync(block_table_dev, block_table_host,
+                           static_cast<size_t>(batch) * block_table_stride * 4,
+                           cudaMemcpyHostToDevice, s)))
+    return e;
+  if ((e = cudaMemcpyAsync(seq_lens_dev, seq_lens_host, static_cast<size_t>(batch) * 4,
+                           cudaMemcpyHostToDevice, s)))
+    return e;
+  if (int rc = kv_append(k_new_dev, v_new_dev, k_cache, v_cache, desc, block_table_dev,
+                         block_table_stride, seq_lens_dev, batch, status, stream))
+    return rc;
+  if (int rc = paged_decode_attention(q_dev, k_cache, v_cache, desc, nullptr, nullptr,
+                                      block_table_dev, block_table_stride, seq_lens_dev, batch,
+                                      num_q_heads, scale, chunk_tokens, out_dev, part_o,
+                                      part_lse, max_chunks, 0u, status, stream))
+    return rc;
+  if (chunk_tokens > 0) {
+    if (int rc = paged_decode_reduce(part_o, part_lse, seq_lens_dev, batch, num_q_heads,
+                                     p.geom.head_dim, chunk_tokens, max_chunks, out_dev, stream))
+      return rc;
+  }
+  if ((e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, s))) return e;
+  return PDA_OK;
+}
+
+int pda_debug_e4m3_decode(float* out256, pda_stream_t stream) {
+  if (!out256) return PDA_ERR_INVALID_ARG;
+  return static_cast<int>(pda::launch_e4m3_decode(out256, static_cast<cudaStream_t>(stream)));
+}
+
+}  // extern "C"

@@ -1,0 +1,78 @@
+// Shared device helpers and the internal launcher interface of libpda.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pda.h"
+
+namespace pda {
+
+constexpr int kPageSize = 16;
+
+// Geometry handed to every kernel by value.
+struct CacheGeom {
+  int64_t page_stride, head_stride, slot_stride;  // elements
+  int32_t num_pages, num_kv_heads, head_dim, dtype;
+};
+
+struct AttnParams {
+  const __nv_bfloat16* q;
+  const void* k_cache;
+  const void* v_cache;
+  const float* k_scale;
+  const float* v_scale;
+  const int32_t* block_table;
+  const int32_t* seq_lens;
+  __nv_bfloat16* out;
+  float* part_o;
+  float* part_lse;
+  int32_t* status;
+  CacheGeom geom;
+  int32_t block_table_stride, batch, num_q_heads, group;  // group = Hq / Hkv
+  int32_t chunk_tokens, max_chunks;
+  float scale;
+};
+
+__device__ __forceinline__ void report(int32_t* status, int code) {
+  if (status != nullptr) atomicMax(status, code);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t bits) {
+  return __uint_as_float(static_cast<uint32_t>(bits) << 16);
+}
+
+// E4M3 byte -> float from the bit fields: exponent 0 is subnormal (m * 2^-9),
+// S.1111.111 is NaN, everything else (1 + m/8) * 2^(e-7).
+__device__ __forceinline__ float e4m3_to_float(uint8_t byte) {
+  const uint32_t sign = static_cast<uint32_t>(byte & 0x80) << 24;
+  const uint32_t e = (byte >> 3) & 0xF;
+  const uint32_t m = byte & 0x7;
+  uint32_t bits;
+  if (e == 0xF && m == 0x7) {
+    bits = 0x7FC00000u;
+  } else if (e == 0) {
+    bits = __float_as_uint(static_cast<float>(m) * 0.001953125f);
+  } else {
+    bits = ((e + 120u) << 23) | (m << 20);
+  }
+  return __uint_as_float(bits | sign);
+}
+
+// Launchers (each returns the cudaError_t of its launch).
+cudaError_t launch_kv_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                             const CacheGeom& g, const int32_t* block_table, int32_t bt_stride,
+                             const int32_t* seq_lens, int32_t batch, int32_t* status,
+                             cudaStream_t stream);
+cudaError_t launch_attention_generic(const AttnParams& p, cudaStream_t stream);
+// Returns cudaErrorNotSupported when the shape is outside the fast kernel's set.
+cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream);
+bool attention_tma_supports(const AttnParams& p);
+cudaError_t launch_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
+                          int32_t batch, int32_t num_q_heads, int32_t head_dim,
+                          int32_t chunk_tokens, int32_t max_chunks, __nv_bfloat16* out,
+                          cudaStream_t stream);
+cudaError_t launch_e4m3_decode(float* out256, cudaStream_t stream);
+
+}  // namespace pda

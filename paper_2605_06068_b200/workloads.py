@@ -8,8 +8,9 @@ oracle's callers: both receive the very same host arrays.
 bf16 tensors are carried as ``uint16`` bit patterns, e4m3 tensors as ``uint8``.
 
 Recipe common to all workloads (one ``numpy.random.Generator(PCG64(seed))``,
-draws in this order): lengths -> page permutation -> q -> K, V (page by page in
-physical-page order of use) -> k_new, v_new. Values are N(0,1) rounded to bf16
+draws in this order): lengths -> page permutation -> q -> K, V (pages in order of
+first use, in slabs of 1024 pages, slab s from the s-th spawned child generator)
+-> k_new, v_new. Values are N(0,1) rounded to bf16
 (round to nearest even). ``seq_lens`` is the length AFTER this step's append;
 the caches hold tokens ``0 .. L-2`` and the slot of token ``L-1`` is poisoned
 until ``kv_append`` writes ``k_new``/``v_new`` there. Physical pages come from a
@@ -38,7 +39,11 @@ BASE_SEED = 42  # the seed the paper's load generator uses (Appendix A, Scenario
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """float32 -> bf16 bit patterns, round to nearest even (finite inputs)."""
-    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    if x.size >= (1 << 16):  # library cast (same rounding), multi-threaded
+        import torch
+        return torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    u = x.view(np.uint32)
     r = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
     return ((u + r) >> np.uint32(16)).astype(np.uint16)
 
@@ -110,13 +115,27 @@ def _deal_pages(rng, pages_per_seq, shared_prefix_pages=0):
     return table, pool
 
 
-def _fill_normal_bf16(rng, dst_u16_2d, rows_idx, slab=2048):
-    """dst[rows_idx[i]] = bf16(N(0,1)) row by row, drawn in slabs to bound memory."""
+def _fill_normal_bf16(rng, dst_u16_2d, rows_idx, slab=1024):
+    """dst[rows_idx[i]] = bf16(N(0,1)). Rows are cut into slabs of ``slab`` rows;
+    slab s is drawn from the s-th child generator spawned from ``rng`` (so the
+    result does not depend on how many threads fill the slabs)."""
     width = dst_u16_2d.shape[1]
-    for s in range(0, len(rows_idx), slab):
-        idx = rows_idx[s:s + slab]
-        x = rng.standard_normal((len(idx), width), dtype=np.float32)
+    starts = list(range(0, len(rows_idx), slab))
+    children = rng.spawn(len(starts)) if starts else []
+
+    def work(i):
+        idx = rows_idx[starts[i]:starts[i] + slab]
+        x = children[i].standard_normal((len(idx), width), dtype=np.float32)
         dst_u16_2d[idx] = f32_to_bf16_bits(x)
+
+    if len(starts) <= 1:
+        for i in range(len(starts)):
+            work(i)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        import os
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+            list(ex.map(work, range(len(starts))))
 
 
 def make_workload(name, seq_lens, num_q_heads, num_kv_heads, head_dim, page_size=16,
@@ -144,8 +163,11 @@ def make_workload(name, seq_lens, num_q_heads, num_kv_heads, head_dim, page_size
                 used.append(int(p))
     used = np.asarray(used, dtype=np.int64)
     tile = Hkv * P * D
-    kb = np.full((num_pages, tile), 0xFFFF, dtype=np.uint16)
-    vb = np.full((num_pages, tile), 0xFFFF, dtype=np.uint16)
+    kb = np.empty((num_pages, tile), dtype=np.uint16)
+    vb = np.empty((num_pages, tile), dtype=np.uint16)
+    unused = np.setdiff1d(np.arange(num_pages, dtype=np.int64), used)
+    kb[unused] = 0xFFFF
+    vb[unused] = 0xFFFF
     _fill_normal_bf16(rng, kb, used)
     _fill_normal_bf16(rng, vb, used)
     if value_scale != 1.0:

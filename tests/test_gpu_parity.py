@@ -1,0 +1,346 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle on
+the same seeded inputs. Integer / byte work is compared bit-exactly, floating
+point within |err| <= atol + rtol*|ref| with (5e-3, 1e-2) for bf16 KV and
+(2e-2, 2e-2) for e4m3 KV, plus a normalised-error gate (see util.py)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_06068_b200 import binding as pda
+from paper_2605_06068_b200 import workloads as W
+
+from util import (DeviceWorkload, assert_close, bf16_tensor, bf16_to_bits, bf16_to_f64,
+                  host_appended, oracle_out)
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [pytest.param(0, id="fast"), pytest.param(pda.PDA_FLAG_FORCE_GENERIC, id="generic")]
+
+
+def status_of(dw):
+    return int(dw.status.item())
+
+
+# ---- kv_append ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("seed", [42, 43, 44, 45])
+def test_kv_append_bit_exact_whole_cache(oracle, seed):
+    w = W.tiny(seed=seed)
+    dw = DeviceWorkload(w)
+    dw.append()
+    k_ref, v_ref = host_appended(oracle, w)
+    assert (bf16_to_bits(dw.k_cache) == k_ref).all()
+    assert (bf16_to_bits(dw.v_cache) == v_ref).all()
+    assert status_of(dw) == 0
+
+
+def test_kv_append_strided_cache_and_guard_regions(oracle):
+    """[pages, slot, head, D] storage viewed as [pages, head, slot, D]; sentinel bytes
+    around the cache must survive."""
+    w = W.make_workload("nhd", [1, 16, 17, 250], 4, 4, 128, seed=5)
+    k_ref, v_ref = host_appended(oracle, w)
+    guard = 4096
+    n = w.k_cache.size
+    bufs = []
+    for host in (w.k_cache, w.v_cache):
+        raw = torch.full((n + 2 * guard,), -21555, dtype=torch.int16, device="cuda")
+        body = raw[guard:guard + n].view(w.num_pages, 16, w.num_kv_heads, w.head_dim)
+        body.copy_(torch.from_numpy(host.view(np.int16)).cuda().permute(0, 2, 1, 3))
+        bufs.append((raw, body.permute(0, 2, 1, 3).view(torch.bfloat16)))
+    dw = DeviceWorkload(w)
+    pda.kv_append(dw.k_new, dw.v_new, bufs[0][1], bufs[1][1], dw.block_table, dw.seq_lens,
+                  status=dw.status)
+    assert (bf16_to_bits(bufs[0][1]) == k_ref).all() and (bf16_to_bits(bufs[1][1]) == v_ref).all()
+    for raw, _ in bufs:
+        assert (raw[:guard] == -21555).all() and (raw[-guard:] == -21555).all()
+    # attention through the same strided view
+    out = pda.paged_decode_attention(dw.q, bufs[0][1], bufs[1][1], dw.block_table, dw.seq_lens,
+                                     float(w.scale), status=dw.status)
+    assert_close(bf16_to_f64(out), oracle_out(oracle, w, k_ref, v_ref), what="strided")
+    assert status_of(dw) == 0
+
+
+def test_kv_append_bad_inputs_set_status_and_touch_nothing(oracle):
+    w = W.tiny(seed=42)
+    dw = DeviceWorkload(w)
+    before_k = bf16_to_bits(dw.k_cache).copy()
+    bt = dw.block_table.clone()
+    bt[0, 1] = w.num_pages          # row 0 appends into logical page 1 (L=17)
+    bt[1, 2] = -1                   # row 1 appends into logical page 2 (L=33)
+    sl = dw.seq_lens.clone()
+    sl[3] = bt.shape[1] * 16 + 1    # beyond the table
+    pda.kv_append(dw.k_new, dw.v_new, dw.k_cache, dw.v_cache, bt, sl, status=dw.status)
+    torch.cuda.synchronize()
+    assert status_of(dw) == 2       # the larger of BAD_PAGE (1) and BAD_SEQ_LEN (2)
+    after = bf16_to_bits(dw.k_cache)
+    # only row 2 (L=64) was appended
+    page = w.block_table[2, 3]
+    expect = before_k.copy()
+    expect[page, :, 15, :] = w.k_new[2]
+    assert (after == expect).all()
+
+
+# ---- attention: tiny config and small ragged cases ----------------------------------------
+
+@pytest.mark.parametrize("flags", PATHS)
+@pytest.mark.parametrize("seed", [42, 43, 44, 45])
+def test_tiny_unsplit_and_split(oracle, seed, flags):
+    w = W.tiny(seed=seed)
+    dw = DeviceWorkload(w)
+    dw.append()
+    ref = oracle_out(oracle, w)
+    out = dw.attend(flags=flags)
+    assert_close(bf16_to_f64(out), ref, what="tiny unsplit")
+    for chunk in (16, 32, 48, 128):
+        out_s = dw.attend(chunk_tokens=chunk, flags=flags)
+        assert_close(bf16_to_f64(out_s), ref, what=f"tiny chunk {chunk}")
+        # partials themselves against the oracle's per-chunk results
+        k, v = host_appended(oracle, w)
+        mc = dw.part_o.shape[2]
+        po, pl = oracle.paged_decode_attention(w.q, k, v, w.block_table, w.seq_lens, w.scale,
+                                               chunk_tokens=chunk, max_chunks=mc)
+        live = ~np.isnan(pl)
+        g_po, g_pl = dw.part_o.cpu().numpy().astype(np.float64), dw.part_lse.cpu().numpy().astype(np.float64)
+        assert np.isnan(g_pl[~live]).all(), "entries of chunks that do not exist must stay untouched"
+        np.testing.assert_allclose(g_pl[live], pl[live], rtol=0, atol=2e-3)
+        assert np.abs(g_po[live] - po[live]).max() < 5e-3
+    assert status_of(dw) == 0
+
+
+RAGGED = [
+    # (lengths, Hq, Hkv, D)
+    ([1, 2, 15, 16, 17, 31, 32, 33, 255, 256, 257, 1000], 8, 2, 64),
+    ([1, 16, 17, 129, 640, 2049], 32, 8, 128),
+    ([5, 48, 300, 777], 64, 8, 128),     # G = 8
+    ([3, 100, 513], 8, 8, 128),          # G = 1
+    ([7, 64, 200], 6, 3, 64),            # G = 2
+    ([9, 130], 24, 2, 96),               # G = 12, head_dim 96: generic kernel only
+]
+
+
+@pytest.mark.parametrize("flags", PATHS)
+@pytest.mark.parametrize("case", RAGGED, ids=lambda c: f"Hq{c[1]}kv{c[2]}D{c[3]}")
+def test_ragged_batches(oracle, case, flags):
+    lens, Hq, Hkv, D = case
+    w = W.make_workload("ragged", lens, Hq, Hkv, D, seed=77)
+    dw = DeviceWorkload(w)
+    dw.append()
+    ref = oracle_out(oracle, w)
+    assert_close(bf16_to_f64(dw.attend(flags=flags)), ref, what="ragged unsplit")
+    for chunk in (64, 512):
+        assert_close(bf16_to_f64(dw.attend(chunk_tokens=chunk, flags=flags)), ref,
+                     what=f"ragged chunk {chunk}")
+    assert status_of(dw) == 0
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_fp8_small(oracle, flags):
+    w = W.prefix_fp8(seed=46, batch=5)
+    dw = DeviceWorkload(w)
+    ref = oracle_out(oracle, w)
+    assert_close(bf16_to_f64(dw.attend(flags=flags)), ref, "e4m3", what="fp8 unsplit")
+    assert_close(bf16_to_f64(dw.attend(chunk_tokens=256, flags=flags)), ref, "e4m3", what="fp8 split")
+    w2 = W.make_workload("fp8r", [1, 15, 16, 17, 100, 333], 16, 2, 64, kv_dtype="e4m3", seed=8)
+    dw2 = DeviceWorkload(w2)
+    assert_close(bf16_to_f64(dw2.attend(flags=flags)), oracle_out(oracle, w2), "e4m3", what="fp8 D64")
+    assert status_of(dw) == 0 and status_of(dw2) == 0
+
+
+def test_e4m3_device_decoder_matches_table(oracle):
+    t = oracle.e4m3_decode_table()
+    g = pda.debug_e4m3_decode().cpu().numpy().astype(np.float64)
+    ok = ~np.isnan(t)
+    assert (g[ok] == t[ok]).all() and np.isnan(g[~ok]).all()
+    assert (np.signbit(g[ok]) == np.signbit(t[ok])).all()
+
+
+# ---- invariants and anti-shortcut checks ---------------------------------------------------
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_single_token_returns_v_bits(oracle, flags):
+    w = W.make_workload("one", [1, 1, 1, 1], 8, 2, 64, seed=3)
+    dw = DeviceWorkload(w)
+    dw.append()
+    out = bf16_to_bits(dw.attend(flags=flags))
+    for b in range(4):
+        for h in range(8):
+            assert (out[b, h] == w.v_new[b, h // 4]).all()
+    w = W.make_workload("one", [1, 1], 32, 8, 128, seed=4)
+    dw = DeviceWorkload(w)
+    dw.append()
+    out = bf16_to_bits(dw.attend(flags=flags))
+    for b in range(2):
+        for h in range(32):
+            assert (out[b, h] == w.v_new[b, h // 4]).all()
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_equal_scores_give_mean_and_empty_sequence_gives_zero(oracle, flags):
+    w = W.make_workload("mean", [0, 40, 700, 0, 16], 32, 8, 128, seed=6)
+    dw = DeviceWorkload(w)
+    dw.append()
+    dw.q.zero_()
+    k, v = host_appended(oracle, w)
+    ref = oracle_out(oracle, type(w)(**{**w.__dict__, "q": np.zeros_like(w.q)}), k, v)
+    for chunk in (0, 128):
+        out = bf16_to_f64(dw.attend(chunk_tokens=chunk, flags=flags))
+        assert (out[0] == 0).all() and (out[3] == 0).all()
+        assert_close(out, ref, what="equal scores")
+        # independent of the oracle: the mean of the gathered V rows
+        L = 700
+        pages = w.block_table[2, :(L + 15) // 16]
+        V = W.bf16_bits_to_f32(v[pages]).astype(np.float64).transpose(1, 0, 2, 3).reshape(8, -1, 128)[:, :L]
+        assert np.abs(out[2, 5] - V[1].mean(axis=0)).max() < 1e-3
+
+
+@pytest.mark.parametrize("flags", PATHS)
+@pytest.mark.parametrize("chunk", [0, 512])
+def test_needle_tokens(oracle, flags, chunk):
+    """One key at score 40 with V = 1..D: a dropped, duplicated or misplaced token shows at O(1)."""
+    L, D = 1500, 128
+    w = W.make_workload("needle", [L], 4, 1, D, seed=13)
+    dw = DeviceWorkload(w)
+    dw.append()
+    q = w.q.copy(); q[0, 1:] = q[0, 0]
+    dw.q = bf16_tensor(q)
+    qf = W.bf16_bits_to_f32(q[0, 0]).astype(np.float64)
+    k0, v0 = dw.k_cache.clone(), dw.v_cache.clone()
+    needle_k = W.f32_to_bf16_bits((40.0 / (float(w.scale) * (qf @ qf)) * qf).astype(np.float32))
+    needle_v = W.f32_to_bf16_bits(np.arange(1, D + 1, dtype=np.float32))
+    for j in (0, 1, 15, 16, 17, 511, 512, 513, 1023, 1024, L - 17, L - 16, L - 2, L - 1):
+        dw.k_cache.copy_(k0); dw.v_cache.copy_(v0)
+        page, slot = int(w.block_table[0, j // 16]), j % 16
+        dw.k_cache[page, 0, slot] = bf16_tensor(needle_k)
+        dw.v_cache[page, 0, slot] = bf16_tensor(needle_v)
+        out = bf16_to_f64(dw.attend(chunk_tokens=chunk, flags=flags))
+        for h in range(4):
+            assert np.abs(out[0, h] - np.arange(1, D + 1)).max() <= 0.5, f"needle at {j}"
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_structured_v(oracle, flags):
+    """V_j[d] = 1 + d/D for every token => out[d] = 1 + d/D (normalisation by l);
+    V_j[0] = j/L => out[0] = sum_j p_j j/L (token <-> weight pairing, via the oracle)."""
+    L, D = 2100, 128
+    w = W.make_workload("sv", [L, 333], 8, 2, D, seed=17, value_scale=3.0)
+    k, v = host_appended(oracle, w)
+    ramp = W.f32_to_bf16_bits(1.0 + np.arange(D, dtype=np.float32) / D)
+    for b, Lb in enumerate((L, 333)):
+        for j in range(Lb):
+            page = w.block_table[b, j // 16]
+            v[page, :, j % 16, :] = ramp
+            v[page, :, j % 16, 0] = W.f32_to_bf16_bits(np.float32(j // 16) / 256)
+    w.k_cache, w.v_cache = k, v
+    w.k_new = np.stack([k[w.block_table[b, (Lb - 1) // 16], :, (Lb - 1) % 16] for b, Lb in enumerate((L, 333))])
+    w.v_new = np.stack([v[w.block_table[b, (Lb - 1) // 16], :, (Lb - 1) % 16] for b, Lb in enumerate((L, 333))])
+    dw = DeviceWorkload(w)
+    ref = oracle_out(oracle, w, k, v)
+    for chunk in (0, 256):
+        out = bf16_to_f64(dw.attend(chunk_tokens=chunk, flags=flags))
+        assert np.abs(out[:, :, 1:] - (1.0 + np.arange(1, D) / D)).max() < 8e-3
+        assert np.abs(out[:, :, 0] - ref[:, :, 0]).max() < 5e-3
+        assert_close(out, ref, what="structured V")
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_page_permutation_poison_and_determinism(oracle, flags):
+    w = W.make_workload("perm", [17, 33, 64, 100, 900], 32, 8, 128, seed=42)
+    dw = DeviceWorkload(w)
+    dw.append()
+    out1 = bf16_to_bits(dw.attend(flags=flags)).copy()
+    out1b = bf16_to_bits(dw.attend(flags=flags))
+    assert (out1 == out1b).all(), "run-to-run determinism"
+    split1 = bf16_to_bits(dw.attend(chunk_tokens=64, flags=flags)).copy()
+    # re-deal the physical pages under a consistent block table
+    rng = np.random.default_rng(1)
+    perm = rng.permutation(w.num_pages)
+    k, v = host_appended(oracle, w)
+    k2 = np.empty_like(k); v2 = np.empty_like(v)
+    k2[perm] = k; v2[perm] = v
+    # change every poison pattern on the way: unused slots, unused pages, table tail
+    used = np.zeros(w.num_pages, bool)
+    for b in range(w.batch):
+        L = int(w.seq_lens[b]); n = (L + 15) // 16
+        used[perm[w.block_table[b, :n]]] = True
+        if L % 16:
+            k2[perm[w.block_table[b, n - 1]], :, L % 16:, :] = 0x7F80   # +inf
+            v2[perm[w.block_table[b, n - 1]], :, L % 16:, :] = 0x7FC0   # NaN
+    k2[~used] = 0x7F80; v2[~used] = 0xFF80
+    table2 = np.where(w.block_table >= 0, perm[np.maximum(w.block_table, 0)], 2 ** 31 - 1).astype(np.int32)
+    w2 = type(w)(**{**w.__dict__, "k_cache": k2, "v_cache": v2, "block_table": table2})
+    dw2 = DeviceWorkload(w2)
+    out2 = bf16_to_bits(dw2.attend(flags=flags))
+    assert (out2 == out1).all(), "page placement and poison must not change a single bit"
+    assert (bf16_to_bits(dw2.attend(chunk_tokens=64, flags=flags)) == split1).all()
+    assert status_of(dw) == 0 and status_of(dw2) == 0
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_bad_block_table_sets_status_and_zero_fills(oracle, flags):
+    w = W.make_workload("bad", [100, 200, 300], 8, 2, 64, seed=9)
+    dw = DeviceWorkload(w)
+    dw.append()
+    good = bf16_to_bits(dw.attend(flags=flags)).copy()
+    guard_q = dw.q.clone()
+    dw.block_table[0, 3] = -1
+    dw.block_table[1, 0] = w.num_pages
+    out = bf16_to_bits(dw.attend(flags=flags))
+    torch.cuda.synchronize()
+    assert status_of(dw) == 1
+    assert (out[0] == 0).all() and (out[1] == 0).all() and (out[2] == good[2]).all()
+    assert torch.equal(dw.q, guard_q)
+    dw.status.zero_()
+    dw.seq_lens[2] = dw.block_table.shape[1] * 16 + 5
+    out = bf16_to_bits(dw.attend(chunk_tokens=64, flags=flags, max_chunks=8))
+    torch.cuda.synchronize()
+    assert status_of(dw) == 2
+    assert (out[2] == 0).all()
+
+
+# ---- reduce on synthetic partials ----------------------------------------------------------
+
+def test_reduce_alone(oracle):
+    rng = np.random.default_rng(0)
+    B, Hq, Cm, D = 3, 8, 7, 128
+    po = rng.standard_normal((B, Hq, Cm, D)).astype(np.float32)
+    pl = (rng.standard_normal((B, Hq, Cm)) * 3).astype(np.float32)
+    seq = np.array([7 * 32, 33, 0], np.int32)
+    po[1, :, 2:] = np.nan; pl[1, :, 2:] = np.nan   # chunks that do not exist: never read
+    ref, _ = oracle.paged_decode_reduce(po.astype(np.float64), pl.astype(np.float64), seq, 32)
+    out = pda.paged_decode_reduce(torch.from_numpy(po).cuda(), torch.from_numpy(pl).cuda(),
+                                  torch.from_numpy(seq).cuda(), 32)
+    assert_close(bf16_to_f64(out), ref, what="reduce", norm=False)
+    assert (bf16_to_f64(out)[2] == 0).all()
+    # a single chunk is the identity (up to the bf16 rounding of the output)
+    out1 = pda.paged_decode_reduce(torch.from_numpy(po).cuda(), torch.from_numpy(pl).cuda(),
+                                   torch.tensor([5, 32, 1], dtype=torch.int32).cuda(), 32)
+    expect = torch.from_numpy(po[:, :, 0]).to(torch.bfloat16)
+    assert torch.equal(out1.cpu(), expect)
+
+
+# ---- the end-to-end host call ---------------------------------------------------------------
+
+def test_step_host_matches_device_calls(oracle):
+    w = W.make_workload("host", [17, 33, 64, 100, 1200], 32, 8, 128, seed=42)
+    dw = DeviceWorkload(w)
+    ref = oracle_out(oracle, w)
+    pin = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+    hq, hk, hv = pin(w.q), pin(w.k_new), pin(w.v_new)
+    hbt, hsl = pin(w.block_table), pin(w.seq_lens)
+    dq, dk, dv = torch.empty_like(dw.q), torch.empty_like(dw.k_new), torch.empty_like(dw.v_new)
+    dbt, dsl = torch.empty_like(dw.block_table), torch.empty_like(dw.seq_lens)
+    for chunk in (0, 256):
+        dw = DeviceWorkload(w)
+        mc = pda.max_chunks(1200, chunk) if chunk else 0
+        po = torch.empty((w.batch, 32, mc, 128), dtype=torch.float32, device="cuda") if chunk else None
+        pl = torch.empty((w.batch, 32, mc), dtype=torch.float32, device="cuda") if chunk else None
+        out_dev = torch.empty_like(dw.q)
+        out_host = torch.zeros(w.q.shape, dtype=torch.int16).pin_memory()
+        pda.paged_decode_step_host(hq.view(torch.bfloat16), hk, hv, hbt, hsl, dq, dk, dv, dbt, dsl,
+                                   dw.k_cache, dw.v_cache, float(w.scale), chunk, po, pl,
+                                   out_dev, out_host, status=dw.status)
+        torch.cuda.synchronize()
+        got = W.bf16_bits_to_f32(out_host.numpy().view(np.uint16)).astype(np.float64)
+        assert_close(got, ref, what=f"step_host chunk {chunk}")
+        k_ref, _ = host_appended(oracle, w)
+        assert (bf16_to_bits(dw.k_cache) == k_ref).all()
