@@ -36,7 +36,9 @@ __global__ void __launch_bounds__(32) attention_generic_kernel(AttnParams p) {
     if (t0 >= L) return;  // no such chunk
     t1 = min(t0 + p.chunk_tokens, L);
   }
-  const bool too_long = static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize;
+  const bool too_long =
+      static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
+      (split && static_cast<int64_t>(L) > static_cast<int64_t>(p.max_chunks) * p.chunk_tokens);
 
   __shared__ float q_s[256];
   for (int d = lane; d < D; d += 32) q_s[d] = __bfloat162float(p.q[row * D + d]);
@@ -107,14 +109,14 @@ __global__ void __launch_bounds__(32) attention_generic_kernel(AttnParams p) {
 #pragma unroll
     for (int i = 0; i < kMaxDPerLane; ++i) {
       const int d = lane + 32 * i;
-      if (d < D) p.part_o[pr * D + d] = acc[i] * inv_l;
+      if (d < D) p.part_o[pr * D + d] = failed ? 0.f : acc[i] * inv_l;
     }
     if (lane == 0) p.part_lse[pr] = (l > 0.f && !failed) ? m + logf(l) : -INFINITY;
   } else {
 #pragma unroll
     for (int i = 0; i < kMaxDPerLane; ++i) {
       const int d = lane + 32 * i;
-      if (d < D) p.out[row * D + d] = __float2bfloat16_rn(acc[i] * inv_l);
+      if (d < D) p.out[row * D + d] = __float2bfloat16_rn(failed ? 0.f : acc[i] * inv_l);
     }
   }
 }

@@ -1,7 +1,528 @@
-// TMA + tensor-core paged decode attention (placeholder until the kernel lands).
+// Paged decode attention for sm_100a: TMA page gather + tensor-core GQA tiles.
+//
+// Work item = (sequence b, kv head g, chunk c) = one CTA of kWarps warps. Every
+// warp is a self-contained flash-decoding worker: it owns a ring of kStages
+// shared-memory stages, each one (page, kv head) K tile plus V tile, filled by
+// 5-D tiled TMA copies (128-byte swizzle) that complete on the warp's own
+// mbarriers, so the steady state has no CTA-wide synchronisation. Warp w takes
+// the chunk's pages w, w+kWarps, ...; the warps' (m, l, O) states are merged
+// through shared memory once at the end.
+//
+// Per 16-token page tile, with the G <= 8 query heads of the group as the N
+// dimension of mma.sync.m16n8k16 (tokens are M, so a page is exactly one MMA
+// row block and nothing is padded along the streamed dimension):
+//   S^T[16 x 8]  = K_tile[16 x D] . Q_g^T[D x 8]          (D/16 MMAs)
+//   online softmax over tokens (max by shuffles across the 8 row groups)
+//   O^T[D x 8]  += V_tile^T[D x 16] . P^T[16 x 8]          (D/16 MMAs)
+// K fragments come from ldmatrix, V^T fragments from ldmatrix.trans, P^T is
+// turned from accumulator layout into B-operand layout by movmatrix. e4m3 tiles
+// are converted to f16 in registers (cvt.rn.f16x2.e4m3x2, exact); their
+// per-(page, head) scales multiply the scores (K) and the probabilities (V).
+//
+// Every wait on an mbarrier is bounded; on expiry the CTA reports
+// PDA_DEV_TIMEOUT, waits (bounded) for its copies in flight and zero-fills its
+// output. TMA copies never use multicast.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace pda {
-bool attention_tma_supports(const AttnParams&) { return false; }
-cudaError_t launch_attention_tma(const AttnParams&, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kWarps = 4;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+// ---- PTX wrappers ------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kSpinLimit polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+template <bool kF16>
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  if (kF16) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+  } else {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+  }
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// (lo, hi) fp32 -> packed 16-bit pair, lo in bits 0..15
+template <bool kF16>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  uint32_t r;
+  if (kF16) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// two e4m3 bytes (bits 0..15 of x) -> f16x2
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
+  uint32_t r;
+  asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, t;\n\t}" : "=r"(r) : "r"(x));
+  return r;
+}
+
+// ---- kernel ------------------------------------------------------------------------------
+
+template <int D, bool kFp8, int kStages>
+struct Cfg {
+  static constexpr int kElem = kFp8 ? 1 : 2;
+  static constexpr int kRowBytes = D * kElem;            // one token row
+  static constexpr int kTileBytes = kPageSize * kRowBytes;
+  static constexpr int kStageBytes = 2 * kTileBytes;     // K tile then V tile
+  static constexpr int kWarpRing = kStages * kStageBytes;
+  static constexpr int kKSteps = D / 16;                 // MMAs of each product per tile
+  static constexpr int kOStride = D + 4;                 // fp32 row pitch of the merge buffer
+  static constexpr int kMergeBytes = (8 * kOStride + 16) * 4;
+  static constexpr int kSmemBytes = kWarps * kWarpRing + kWarps * kStages * 8 + 16 + 1024;
+  static_assert(kRowBytes % 128 == 0, "rows must be whole 128-byte swizzle lines");
+  static_assert(kMergeBytes <= kWarpRing, "merge buffer reuses the warp's ring");
+};
+
+// Byte offset of 16-byte chunk `chunk` of row `r` inside a tile stored as kSub
+// sub-tiles of [16 rows][128 B] with the 128-byte TMA swizzle.
+__device__ __forceinline__ uint32_t tile_off(int r, int chunk) {
+  return static_cast<uint32_t>((chunk >> 3) * (kPageSize * 128) + r * 128 + (((chunk & 7) ^ (r & 7)) << 4));
+}
+
+template <int D, bool kFp8, int kStages>
+__global__ void __launch_bounds__(kWarps * 32)
+attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
+                     const __grid_constant__ CUtensorMap v_map, AttnParams p) {
+  using C = Cfg<D, kFp8, kStages>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kWarps * C::kWarpRing);
+  int* cta_err = reinterpret_cast<int*>(bars + kWarps * kStages);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int gid = lane >> 2, tq = lane & 3;
+  const int c = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int G = p.group;
+  const bool split = p.chunk_tokens > 0;
+  const int64_t row0 = static_cast<int64_t>(b) * p.num_q_heads + static_cast<int64_t>(g) * G;
+
+  const int L = max(p.seq_lens[b], 0);
+  int t0 = 0, t1 = L;
+  if (split) {
+    t0 = c * p.chunk_tokens;
+    if (t0 >= L) return;
+    t1 = min(t0 + p.chunk_tokens, L);
+  }
+  int err = 0;
+  if (static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
+      (split && static_cast<int64_t>(L) > static_cast<int64_t>(p.max_chunks) * p.chunk_tokens))
+    err = PDA_DEV_BAD_SEQ_LEN;
+
+  if (tid == 0) *cta_err = 0;
+  const int n_tiles = err ? 0 : (t1 - t0 + kPageSize - 1) / kPageSize;
+  const int n_mine = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;  // tiles warp, warp+kWarps, ...
+  const int page0 = t0 / kPageSize;
+
+  const uint32_t ring = smem_u32(smem + warp * C::kWarpRing);
+  const uint32_t bar0 = smem_u32(bars + warp * kStages);
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+    fence_mbar_init();
+    fence_proxy_async();
+  }
+  __syncthreads();  // also orders the cta_err reset
+
+  // ---- page ids (and e4m3 scales) for this warp's tiles, 32 ordinals per register block
+  const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
+  bool bad_page = false;
+  auto load_block = [&](int blk, int& pg, float& ks, float& vs) {
+    const int kk = blk * 32 + lane;
+    pg = 0; ks = 0.f; vs = 0.f;
+    if (kk < n_mine) {
+      const int v = table[page0 + warp + kk * kWarps];
+      if (v < 0 || v >= p.geom.num_pages) bad_page = true; else pg = v;
+      if (kFp8) {
+        ks = p.k_scale[static_cast<int64_t>(pg) * p.geom.num_kv_heads + g];
+        vs = p.v_scale[static_cast<int64_t>(pg) * p.geom.num_kv_heads + g];
+      }
+    }
+  };
+  int pgA, pgB; float ksA, ksB, vsA, vsB;
+  load_block(0, pgA, ksA, vsA);
+  load_block(1, pgB, ksB, vsB);
+
+  auto issue = [&](int kk, int page) {  // lane 0 only
+    const int s = kk % kStages;
+    const uint32_t bar = bar0 + 8 * s;
+    const uint32_t dst = ring + s * C::kStageBytes;
+    mbar_expect_tx(bar, C::kStageBytes);
+    tma_load_5d(dst, &k_map, bar, 0, 0, 0, g, page);
+    tma_load_5d(dst + C::kTileBytes, &v_map, bar, 0, 0, 0, g, page);
+  };
+
+  // prologue: fill the ring
+  {
+    const int n_pre = min(kStages, n_mine);
+    for (int kk = 0; kk < n_pre; ++kk) {
+      const int page = __shfl_sync(0xffffffffu, pgA, kk);
+      if (lane == 0) issue(kk, page);
+    }
+  }
+
+  // ---- Q^T fragments (B operand of S^T = K.Q^T): column n = gid is head gid of the group
+  uint32_t qf[C::kKSteps][2];
+  {
+    const __nv_bfloat16* qrow = p.q + (row0 + gid) * D;
+#pragma unroll
+    for (int ks = 0; ks < C::kKSteps; ++ks) {
+      qf[ks][0] = 0u; qf[ks][1] = 0u;
+      if (gid < G) {
+        if (!kFp8) {
+          qf[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq);
+          qf[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq + 8);
+        } else {
+          // e4m3 K fragments carry d = 16ks+4tq+{0,1} in k-slots {2tq,2tq+1} and
+          // d = 16ks+4tq+{2,3} in k-slots {2tq+8,2tq+9}; q follows the same order.
+          const uint2 raw = *reinterpret_cast<const uint2*>(qrow + 16 * ks + 4 * tq);
+          const float q0 = __uint_as_float(raw.x << 16), q1 = __uint_as_float(raw.x & 0xffff0000u);
+          const float q2 = __uint_as_float(raw.y << 16), q3 = __uint_as_float(raw.y & 0xffff0000u);
+          qf[ks][0] = pack2<true>(q0, q1);
+          qf[ks][1] = pack2<true>(q2, q3);
+        }
+      }
+    }
+  }
+
+  const float scale_log2 = p.scale * 1.4426950408889634f;
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2tq, 2tq+1
+  float o[C::kKSteps][4];
+#pragma unroll
+  for (int i = 0; i < C::kKSteps; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+
+  // ldmatrix lane addressing: matrix j = lane/8, row-in-matrix = lane%8
+  const int lj = lane >> 3, lr = lane & 7;
+  const int k_row = lr + 8 * (lj & 1), k_chk = lj >> 1;        // K (and e4m3 V): rows by j&1, chunk by j>>1
+  const int v_row = kFp8 ? k_row : lr + 8 * (lj >> 1);         // bf16 V^T: rows by j>>1, chunk by j&1
+  const int v_chk = kFp8 ? k_chk : (lj & 1);
+
+  bool timed_out = false;
+  int kk = 0;
+  for (; kk < n_mine; ++kk) {
+    const int s = kk % kStages;
+    const uint32_t bar = bar0 + 8 * s;
+    if (!mbar_wait_bounded(bar, (kk / kStages) & 1)) { timed_out = true; break; }
+    const uint32_t kt = ring + s * C::kStageBytes, vt = kt + C::kTileBytes;
+    const int tok0 = t0 + (warp + kk * kWarps) * kPageSize;
+    const int n_valid = min(kPageSize, t1 - tok0);
+    float ksc = 1.f, vsc = 1.f;
+    if (kFp8) {
+      ksc = __shfl_sync(0xffffffffu, ksA, kk & 31);
+      vsc = __shfl_sync(0xffffffffu, vsA, kk & 31);
+    }
+
+    if (n_valid < kPageSize) {
+      // rows past the sequence end may hold anything: clear them in V (K is masked by select)
+      const int n_chunks = C::kRowBytes / 16;
+      for (int i = lane; i < (kPageSize - n_valid) * n_chunks; i += 32) {
+        const int r = n_valid + i / n_chunks, ch = i % n_chunks;
+        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_off(r, ch)), "r"(0));
+      }
+      __syncwarp();
+    }
+
+    // ---- S^T = K . Q^T
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+    if (!kFp8) {
+#pragma unroll
+      for (int ks = 0; ks < C::kKSteps; ++ks) {
+        uint32_t a[4];
+        ldsm_x4(kt + tile_off(k_row, 2 * ks + k_chk), a);
+        if (ks & 1) mma16816<false>(sb, a, qf[ks][0], qf[ks][1]);
+        else mma16816<false>(sa, a, qf[ks][0], qf[ks][1]);
+      }
+    } else {
+#pragma unroll
+      for (int ks = 0; ks < C::kKSteps; ks += 2) {
+        uint32_t r[4], a[4];
+        ldsm_x4(kt + tile_off(k_row, ks + k_chk), r);   // r0,r1: chunk ks rows 0-7 / 8-15; r2,r3: chunk ks+1
+        a[0] = e4m3x2_to_f16x2(r[0]); a[2] = e4m3x2_to_f16x2(r[0] >> 16);
+        a[1] = e4m3x2_to_f16x2(r[1]); a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+        mma16816<true>(sa, a, qf[ks][0], qf[ks][1]);
+        a[0] = e4m3x2_to_f16x2(r[2]); a[2] = e4m3x2_to_f16x2(r[2] >> 16);
+        a[1] = e4m3x2_to_f16x2(r[3]); a[3] = e4m3x2_to_f16x2(r[3] >> 16);
+        mma16816<true>(sb, a, qf[ks + 1][0], qf[ks + 1][1]);
+      }
+    }
+    const float sc = scale_log2 * ksc;
+    float s0 = (sa[0] + sb[0]) * sc, s1 = (sa[1] + sb[1]) * sc;   // token gid,   heads 2tq, 2tq+1
+    float s2 = (sa[2] + sb[2]) * sc, s3 = (sa[3] + sb[3]) * sc;   // token gid+8
+    if (n_valid < kPageSize) {
+      if (gid >= n_valid) { s0 = -INFINITY; s1 = -INFINITY; }
+      if (gid + 8 >= n_valid) { s2 = -INFINITY; s3 = -INFINITY; }
+    }
+
+    // ---- online softmax (base 2), max over the tile's tokens = over gid and the two rows
+    float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+    }
+    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: token 0 of a tile is always valid
+    const float al0 = ex2(m0 - mn0), al1 = ex2(m1 - mn1);     // ex2(-inf) = 0 on the first tile
+    m0 = mn0; m1 = mn1;
+    const float p0 = ex2(s0 - mn0), p1 = ex2(s1 - mn1), p2 = ex2(s2 - mn0), p3 = ex2(s3 - mn1);
+    l0 = fmaf(l0, al0, p0 + p2);
+    l1 = fmaf(l1, al1, p1 + p3);
+    const uint32_t pb0 = movmatrix_trans(pack2<kFp8>(p0 * vsc, p1 * vsc));   // P^T rows: tokens 0-7
+    const uint32_t pb1 = movmatrix_trans(pack2<kFp8>(p2 * vsc, p3 * vsc));   // tokens 8-15
+
+    // ---- O^T = O^T * alpha + V^T . P^T
+#pragma unroll
+    for (int mt = 0; mt < C::kKSteps; ++mt) {
+      o[mt][0] *= al0; o[mt][1] *= al1; o[mt][2] *= al0; o[mt][3] *= al1;
+    }
+    if (!kFp8) {
+#pragma unroll
+      for (int mt = 0; mt < C::kKSteps; ++mt) {
+        uint32_t a[4];
+        ldsm_x4_trans(vt + tile_off(v_row, 2 * mt + v_chk), a);
+        mma16816<false>(o[mt], a, pb0, pb1);
+      }
+    } else {
+#pragma unroll
+      for (int mt = 0; mt < C::kKSteps; mt += 2) {
+        uint32_t r[4], a[4];
+        ldsm_x4_trans(vt + tile_off(v_row, mt + v_chk), r);
+        // a transposed register holds bytes V[2tq][dA], V[2tq][dA+1], V[2tq+1][dA], V[2tq+1][dA+1]
+        // with dA = 16*chunk + 2gid: regroup to (V[2tq][d], V[2tq+1][d]) pairs for d = dA, dA+1
+#pragma unroll
+        for (int i = 0; i < 4; ++i) r[i] = __byte_perm(r[i], 0, 0x3120);
+        a[0] = e4m3x2_to_f16x2(r[0]); a[1] = e4m3x2_to_f16x2(r[0] >> 16);
+        a[2] = e4m3x2_to_f16x2(r[1]); a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+        mma16816<true>(o[mt], a, pb0, pb1);
+        a[0] = e4m3x2_to_f16x2(r[2]); a[1] = e4m3x2_to_f16x2(r[2] >> 16);
+        a[2] = e4m3x2_to_f16x2(r[3]); a[3] = e4m3x2_to_f16x2(r[3] >> 16);
+        mma16816<true>(o[mt + 1], a, pb0, pb1);
+      }
+    }
+
+    // ---- hand the stage back: every lane has consumed its fragments
+    __syncwarp();
+    const int kn = kk + kStages;
+    if (((kk + 1) & 31) == 0) {  // the consumer moves to the next register block
+      pgA = pgB; ksA = ksB; vsA = vsB;
+      load_block((kk + 1) / 32 + 1, pgB, ksB, vsB);
+    }
+    if (kn < n_mine) {
+      // kn lies in the consumer's block or the one after it
+      const bool in_a = (kn >> 5) == ((kk + 1) >> 5);
+      const int page = __shfl_sync(0xffffffffu, in_a ? pgA : pgB, kn & 31);
+      if (lane == 0) {
+        fence_proxy_async();
+        issue(kn, page);
+      }
+    }
+  }
+
+  if (timed_out) {
+    // give the copies still in flight a bounded chance to land before the CTA's memory is reused
+    for (int j = kk; j < min(kk + kStages, n_mine); ++j)
+      mbar_wait_bounded(bar0 + 8 * (j % kStages), (j / kStages) & 1);
+    if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
+  }
+  if (__any_sync(0xffffffffu, bad_page) && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
+
+  // ---- publish this warp's state into its own (drained) ring
+#pragma unroll
+  for (int off = 4; off < 32; off <<= 1) {
+    l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+  }
+  float* mo = reinterpret_cast<float*>(smem + warp * C::kWarpRing);
+  float* mm = mo + 8 * C::kOStride;  // m[8] then l[8]
+  __syncwarp();
+  if (!timed_out) {
+    if (gid == 0) {
+      mm[2 * tq] = m0; mm[2 * tq + 1] = m1;
+      mm[8 + 2 * tq] = l0; mm[8 + 2 * tq + 1] = l1;
+    }
+    if (2 * tq < G) {
+#pragma unroll
+      for (int mt = 0; mt < C::kKSteps; ++mt) {
+        const int d0 = kFp8 ? 16 * mt + 2 * gid : 16 * mt + gid;
+        const int d1 = kFp8 ? d0 + 1 : d0 + 8;
+        mo[(2 * tq) * C::kOStride + d0] = o[mt][0];
+        mo[(2 * tq + 1) * C::kOStride + d0] = o[mt][1];
+        mo[(2 * tq) * C::kOStride + d1] = o[mt][2];
+        mo[(2 * tq + 1) * C::kOStride + d1] = o[mt][3];
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- merge the warps' states and write the unit's result
+  const int dev_err = max(err, *cta_err);
+  if (dev_err && tid == 0) report(p.status, dev_err);
+  constexpr float kLn2 = 0.6931471805599453f;
+  for (int idx = tid; idx < G * D; idx += kWarps * 32) {
+    const int h = idx / D, d = idx % D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float* wm = reinterpret_cast<const float*>(smem + w * C::kWarpRing) + 8 * C::kOStride;
+      M = fmaxf(M, wm[h]);
+    }
+    float acc = 0.f, lsum = 0.f;
+    if (!dev_err && M > -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const float* wo = reinterpret_cast<const float*>(smem + w * C::kWarpRing);
+        const float* wm = wo + 8 * C::kOStride;
+        const float mw = wm[h];
+        const float wgt = (mw > -INFINITY) ? ex2(mw - M) : 0.f;
+        lsum = fmaf(wm[8 + h], wgt, lsum);
+        if (wgt != 0.f) acc = fmaf(wo[h * C::kOStride + d], wgt, acc);
+      }
+    }
+    const bool live = !dev_err && lsum > 0.f;
+    const float val = live ? acc / lsum : 0.f;
+    if (split) {
+      const int64_t pr = (row0 + h) * p.max_chunks + c;
+      p.part_o[pr * D + d] = val;
+      if (d == 0) p.part_lse[pr] = live ? (M + __log2f(lsum)) * kLn2 : -INFINITY;
+    } else {
+      p.out[(row0 + h) * D + d] = __float2bfloat16_rn(val);
+    }
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                              CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                              CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = [] {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      sym = nullptr;
+    return reinterpret_cast<EncodeFn>(sym);
+  }();
+  return fn;
+}
+
+// 5-D view of a cache: (byte-lane within a 128-byte line, slot, line of the row, head, page).
+bool make_map(CUtensorMap* map, const void* base, const CacheGeom& g) {
+  EncodeFn enc = encode_fn();
+  if (!enc) return false;
+  const int eb = g.dtype == PDA_BF16 ? 2 : 1;
+  const cuuint64_t line_elems = 128 / eb;
+  const cuuint64_t lines = static_cast<cuuint64_t>(g.head_dim) * eb / 128;
+  cuuint64_t dims[5] = {line_elems, static_cast<cuuint64_t>(kPageSize), lines,
+                        static_cast<cuuint64_t>(g.num_kv_heads), static_cast<cuuint64_t>(g.num_pages)};
+  cuuint64_t strides[4] = {static_cast<cuuint64_t>(g.slot_stride) * eb, 128,
+                           static_cast<cuuint64_t>(g.head_stride) * eb,
+                           static_cast<cuuint64_t>(g.page_stride) * eb};
+  cuuint32_t box[5] = {static_cast<cuuint32_t>(line_elems), kPageSize, static_cast<cuuint32_t>(lines), 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  const CUresult r = enc(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 5,
+                         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int D, bool kFp8, int kStages>
+cudaError_t launch(const AttnParams& p, cudaStream_t stream) {
+  using C = Cfg<D, kFp8, kStages>;
+  alignas(64) CUtensorMap k_map, v_map;
+  if (!make_map(&k_map, p.k_cache, p.geom) || !make_map(&v_map, p.v_cache, p.geom))
+    return cudaErrorNotSupported;
+  auto kern = attention_tma_kernel<D, kFp8, kStages>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks) : 1u;
+  dim3 grid(chunks, p.geom.num_kv_heads, p.batch);
+  kern<<<grid, kWarps * 32, C::kSmemBytes, stream>>>(k_map, v_map, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool attention_tma_supports(const AttnParams& p) {
+  if (p.group < 1 || p.group > 8) return false;
+  if (p.geom.num_kv_heads > 65535) return false;
+  if (p.geom.num_pages < 1) return false;
+  if (p.geom.dtype == PDA_BF16) return p.geom.head_dim == 64 || p.geom.head_dim == 128;
+  return p.geom.head_dim == 128;
+}
+
+cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream) {
+  if (p.geom.dtype == PDA_BF16) {
+    if (p.geom.head_dim == 128) return launch<128, false, 3>(p, stream);
+    return launch<64, false, 3>(p, stream);
+  }
+  return launch<128, true, 3>(p, stream);
+}
+
 }  // namespace pda
