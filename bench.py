@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 DEFAULT_CHUNK = {"tiny": 0, "llama8b": 512, "longctx": 2048, "chat70b": 512, "prefix_fp8": 512}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu
 # capture summarised under profiles/ (None: not captured for that workload)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"llama8b": 624_530_000}  # profiles/attention_tma_llama8b_ncu.md
 
 
 def measured_peak():
@@ -110,7 +110,8 @@ def physical_gpu_index(local):
 
 
 def make(name, rank):
-    seed = W.BASE_SEED + list(W.WORKLOADS).index(name) + 1000 * rank
+    from paper_2605_06068_b200.sharding import rank_seed
+    seed = rank_seed(W.BASE_SEED + list(W.WORKLOADS).index(name), rank)
     return W.WORKLOADS[name](seed=seed)
 
 
@@ -271,13 +272,9 @@ def run_gpu(args):
         e2e = (ms_e2e, h2d, d2h)
 
     # ---- aggregate over ranks ----------------------------------------------------------------
-    stats = torch.tensor([ms_step, ms_attn, e2e[0] if e2e else 0.0], dtype=torch.float64, device=dev)
-    sums = torch.tensor([float(w.kv_bytes), float(w.batch)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-        dist.all_reduce(sums, op=dist.ReduceOp.SUM)
-    ms_step, ms_attn, ms_e2e = [float(x) for x in stats.tolist()]
-    kv_bytes_all, batch_all = [float(x) for x in sums.tolist()]
+    from paper_2605_06068_b200.sharding import aggregate
+    (ms_step, ms_attn, ms_e2e), (kv_bytes_all, batch_all) = aggregate(
+        [ms_step, ms_attn, e2e[0] if e2e else 0.0], [float(w.kv_bytes), float(w.batch)], device=dev)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
