@@ -19,8 +19,8 @@
  * Conventions
  *   - All data pointers are DEVICE pointers unless a comment says "host".
  *   - The caller owns every buffer. The library allocates no device memory and
- *     keeps no device state between calls (it memoises TMA descriptors on the
- *     host, keyed by pointer and shape).
+ *     keeps no state between calls (TMA descriptors are rebuilt per call on
+ *     the host and passed by value).
  *   - Every call enqueues work on `stream` (a cudaStream_t passed as void*) and
  *     returns without synchronising. Nothing reads seq_lens or block_table back
  *     to the host, so a step can be captured in a CUDA graph.
@@ -167,6 +167,43 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
                            float scale, int32_t chunk_tokens, float* part_o, float* part_lse,
                            int32_t max_chunks, void* out_dev, void* out_host, int32_t* status,
                            pda_stream_t stream);
+
+/* Split-KV attention plus reduce with library-owned scratch. (The paper has no
+ * counterpart; this entry point exists for integration reasons only.)
+ *
+ * Some callers cannot hand the library partial buffers because they cannot get
+ * device memory when the call is made: a serving process whose start-up code has
+ * already claimed the whole HBM for its KV pool and weights, so that any later
+ * cudaMalloc fails; a plug-in that runs inside a host application's context and
+ * was given no allocator; or a latency-critical loop in which an allocation's
+ * implicit device synchronisation is not acceptable. For them this call does what
+ * paged_decode_attention(chunk_tokens > 0) followed by paged_decode_reduce does,
+ * but keeps part_o / part_lse in a fixed array of PDA_STATIC_SCRATCH_BYTES
+ * compiled into the library's device image. It calls no cudaMalloc, cudaFree or
+ * other allocating routine. Every process that loads the library holds that
+ * array on each GPU it uses, until it exits.
+ *
+ * Arguments are those of paged_decode_attention without the partial buffers and
+ * flags; `out` is [batch, num_q_heads, head_dim] bf16. The sizes must satisfy
+ *   round_up(batch*num_q_heads*max_chunks*head_dim*4, 256)
+ *     + batch*num_q_heads*max_chunks*4  <=  PDA_STATIC_SCRATCH_BYTES,
+ * otherwise PDA_ERR_TOO_LARGE is returned and nothing is enqueued.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current) and caches it; make that first call outside any stream
+ * capture. The array is shared by all calls and keeps the previous call's
+ * contents: nothing in it needs to start at zero (attention writes every entry
+ * that reduce reads), but two calls whose kernels can overlap on the GPU (different
+ * streams, or different host threads without ordering) race on it. Calls on one
+ * stream are ordered and safe. */
+#define PDA_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int paged_decode_attention_static(const void* q, const void* k_cache, const void* v_cache,
+                                  const pda_cache_desc* desc, const float* k_scale,
+                                  const float* v_scale, const int32_t* block_table,
+                                  int32_t block_table_stride, const int32_t* seq_lens,
+                                  int32_t batch, int32_t num_q_heads, float scale,
+                                  int32_t chunk_tokens, int32_t max_chunks, void* out,
+                                  int32_t* status, pda_stream_t stream);
 
 /* Diagnostic: decodes all 256 e4m3 bytes with the device decoder the generic
  * kernel uses; out256: device float[256]. */

@@ -21,7 +21,8 @@ DEV_STATUS = {0: "ok", 1: "bad page id", 2: "seq_len exceeds block table", 3: "c
 
 EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
-           "pda_debug_e4m3_decode"]
+           "pda_debug_e4m3_decode", "paged_decode_attention_static"]
+STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
 class CacheDesc(C.Structure):
@@ -54,6 +55,8 @@ def lib():
         L.paged_decode_step_host.argtypes = [vp] * 5 + [vp] * 5 + [vp, vp, dp, i32, i32, i32, f32,
                                                                  i32, vp, vp, i32, vp, vp, vp, vp]
         L.pda_debug_e4m3_decode.argtypes = [vp, vp]
+        L.paged_decode_attention_static.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32,
+                                                    f32, i32, i32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -162,4 +165,23 @@ def paged_decode_step_host(q_host, k_new_host, v_new_host, block_table_host, seq
 def debug_e4m3_decode(stream=None):
     out = torch.empty(256, dtype=torch.float32, device="cuda")
     _check(lib().pda_debug_e4m3_decode(_ptr(out), _stream(stream)), "pda_debug_e4m3_decode")
+    return out
+
+
+def paged_decode_attention_static(q, k_cache, v_cache, block_table, seq_lens, scale, chunk_tokens,
+                                  max_chunks, out=None, k_scale=None, v_scale=None, status=None,
+                                  stream=None):
+    """Split-KV attention + reduce using the library's built-in scratch array, for
+    callers that cannot allocate partial buffers (see ``include/pda.h``). ``out`` should
+    be passed in by such callers; it is only created here as a convenience. Raises if
+    ``batch*Hq*max_chunks*(D+1)*4`` bytes exceed ``STATIC_SCRATCH_BYTES``."""
+    desc = cache_desc(k_cache)
+    B, Hq, _ = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    rc = lib().paged_decode_attention_static(
+        _ptr(q), _ptr(k_cache), _ptr(v_cache), C.byref(desc), _ptr(k_scale), _ptr(v_scale),
+        _ptr(block_table), block_table.stride(0), _ptr(seq_lens), B, Hq, float(scale),
+        chunk_tokens, max_chunks, _ptr(out), _ptr(status), _stream(stream))
+    _check(rc, "paged_decode_attention_static")
     return out

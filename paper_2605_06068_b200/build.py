@@ -13,7 +13,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libpda.so")
-SOURCES = ["api.cu", "kv_append.cu", "reduce.cu", "attention_generic.cu", "attention_tma.cu"]
+SOURCES = ["api.cu", "kv_append.cu", "reduce.cu", "attention_generic.cu", "attention_tma.cu",
+           "static_scratch.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
