@@ -5,7 +5,8 @@
     python bench.py --impl reference ...      # times the fp64 CPU oracle instead
 
 One "step" = kv_append -> paged_decode_attention (-> paged_decode_reduce) over
-one synthetic decode batch. ``value`` is KV GB/s: algorithmic KV bytes of the
+one synthetic decode batch, by default as the single fused launch
+``paged_decode_step`` (``--path separate`` times the three calls). ``value`` is KV GB/s: algorithmic KV bytes of the
 batch (every valid K and V element once) divided by the step time, inputs
 resident in HBM. Prints ONE JSON line on rank 0. With N > 1 (torchrun) every
 rank runs its own independent batch (sequences shard with no collective), the
@@ -31,7 +32,7 @@ METRIC = "paged decode attention KV GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # chunk_tokens each workload is timed with (longctx is fixed by its definition)
-DEFAULT_CHUNK = {"tiny": 0, "llama8b": 512, "longctx": 2048, "chat70b": 512, "prefix_fp8": 512}
+DEFAULT_CHUNK = {"tiny": 0, "llama8b": 0, "longctx": 2048, "chat70b": 0, "prefix_fp8": 0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu
 # capture summarised under profiles/ (None: not captured for that workload)
 NCU_TRAFFIC_BYTES = {"llama8b": 624_530_000}  # profiles/attention_tma_llama8b_ncu.md
@@ -204,16 +205,28 @@ def run_gpu(args):
         part_o = torch.empty((w.batch, w.num_q_heads, mc, w.head_dim), dtype=torch.float32, device=dev)
         part_lse = torch.empty((w.batch, w.num_q_heads, mc), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
-    launches_per_step = (1 if k_new is not None else 0) + 1 + (1 if chunk else 0)
+    fused = args.path == "fused"
+    workspace = pda.new_workspace(w.batch, w.num_kv_heads, dev)
+    flags = {"tma": 0, "generic": pda.PDA_FLAG_FORCE_GENERIC}[args.kernel]
+    launches_per_step = 1 if fused else (1 if k_new is not None else 0) + 1 + (1 if chunk else 0)
 
     def step(ev=None):
+        if fused:   # append + attention + reduce in one launch
+            if ev:
+                ev[0].record(stream)
+            pda.paged_decode_step(q, k_new, v_new, k_cache, v_cache, bt, sl, float(w.scale),
+                                  chunk_tokens=chunk, out=out, part_o=part_o, part_lse=part_lse,
+                                  workspace=workspace, k_scale=k_scale, v_scale=v_scale, status=status)
+            if ev:
+                ev[1].record(stream)
+            return
         if k_new is not None:
             pda.kv_append(k_new, v_new, k_cache, v_cache, bt, sl, status=status)
         if ev:
             ev[0].record(stream)
         pda.paged_decode_attention(q, k_cache, v_cache, bt, sl, float(w.scale), chunk_tokens=chunk,
                                    out=out, part_o=part_o, part_lse=part_lse, k_scale=k_scale,
-                                   v_scale=v_scale, status=status)
+                                   v_scale=v_scale, flags=flags, status=status)
         if ev:
             ev[1].record(stream)
         if chunk:
@@ -255,7 +268,7 @@ def run_gpu(args):
         def host_step():
             pda.paged_decode_step_host(hq, hk, hv, hbt, hsl, dq, dk, dv, dbt, dsl, k_cache, v_cache,
                                        float(w.scale), chunk, part_o, part_lse, out, out_host,
-                                       status=status)
+                                       workspace=workspace if fused else None, status=status)
         for _ in range(max(args.warmup, 3)):
             host_step()
         barrier()
@@ -286,6 +299,7 @@ def run_gpu(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.kv_dtype == "bf16" else "e4m3",
             "data": "synthetic", "config": config_of(w, chunk, world),
             "tokens_per_s": batch_all / (ms_step * 1e-3),
+            "path": f"{args.path}/{args.kernel}",
             "pct_of_nominal_hbm_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
             "attention_ms": ms_attn,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -321,6 +335,10 @@ def main():
     ap.add_argument("--workload", default="llama8b", choices=list(W.WORKLOADS))
     ap.add_argument("--chunk", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", default="fused", choices=["fused", "separate"],
+                    help="fused: one paged_decode_step launch; separate: kv_append, attention, reduce")
+    ap.add_argument("--kernel", default="tma", choices=["tma", "generic"],
+                    help="attention kernel of the separate path")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -151,10 +151,38 @@ int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_
                         int32_t chunk_tokens, int32_t max_chunks, void* out,
                         pda_stream_t stream);
 
+/* Number of int32 the `workspace` of paged_decode_step needs: 2 + batch*num_kv_heads. */
+int pda_workspace_ints(int32_t batch, int32_t num_kv_heads);
+
+/* One whole decode step of this layer in a single launch: KV append (when k_new
+ * and v_new are given; both NULL skips it), paged decode attention and, for
+ * chunk_tokens > 0, the merge of the split-KV partials -- the three calls above
+ * fused, with the same definitions; `out` [batch, num_q_heads, head_dim] bf16 is
+ * always written. The append is applied to the cache and seen by this step's
+ * attention.
+ *   part_o, part_lse, max_chunks  as in paged_decode_attention (chunk_tokens > 0)
+ *   workspace  device int32[pda_workspace_ints(batch, num_kv_heads)], zeroed by the
+ *              caller ONCE (e.g. at allocation); every call leaves it zeroed again,
+ *              so consecutive calls on one stream may share it. Calls that can
+ *              overlap on the GPU need separate workspaces. It carries the work
+ *              per-(sequence, kv head) chunk counters (two leading ints are
+ *              reserved). May be NULL when chunk_tokens == 0. After a
+ *              PDA_DEV_TIMEOUT status, zero it again.
+ * If chunk_tokens > 0 and workspace is NULL, or the shape is outside the fused
+ * kernel's set (group size > 8, head_dim not 64/128), the step is
+ * run as the separate launches instead, with the same result. */
+int paged_decode_step(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                      void* v_cache, const pda_cache_desc* desc, const float* k_scale,
+                      const float* v_scale, const int32_t* block_table,
+                      int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+                      int32_t num_q_heads, float scale, int32_t chunk_tokens, void* out,
+                      float* part_o, float* part_lse, int32_t max_chunks, int32_t* workspace,
+                      int32_t* status, pda_stream_t stream);
+
 /* One whole decode step driven from HOST buffers (the end-to-end call): copies
  * this step's q, k_new, v_new, seq_lens and block_table from (ideally pinned)
- * host memory into the caller's device staging buffers, runs kv_append,
- * paged_decode_attention and (chunk_tokens > 0) paged_decode_reduce, and copies
+ * host memory into the caller's device staging buffers, runs
+ * paged_decode_step (workspace as described there, may be NULL), and copies
  * `out` back to out_host; all on `stream`, without synchronising. The KV cache
  * itself stays resident on the device between steps. *_dev are device buffers
  * of the same sizes as their host counterparts. */
@@ -165,8 +193,8 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
                            void* k_cache, void* v_cache, const pda_cache_desc* desc,
                            int32_t block_table_stride, int32_t batch, int32_t num_q_heads,
                            float scale, int32_t chunk_tokens, float* part_o, float* part_lse,
-                           int32_t max_chunks, void* out_dev, void* out_host, int32_t* status,
-                           pda_stream_t stream);
+                           int32_t max_chunks, int32_t* workspace, void* out_dev, void* out_host,
+                           int32_t* status, pda_stream_t stream);
 
 /* Split-KV attention plus reduce with library-owned scratch. (The paper has no
  * counterpart; this entry point exists for integration reasons only.)

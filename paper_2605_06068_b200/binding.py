@@ -21,7 +21,8 @@ DEV_STATUS = {0: "ok", 1: "bad page id", 2: "seq_len exceeds block table", 3: "c
 
 EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
-           "pda_debug_e4m3_decode", "paged_decode_attention_static"]
+           "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
+           "paged_decode_step"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
@@ -53,7 +54,10 @@ def lib():
                                              i32, vp, vp, vp, i32, u32, vp, vp]
         L.paged_decode_reduce.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
         L.paged_decode_step_host.argtypes = [vp] * 5 + [vp] * 5 + [vp, vp, dp, i32, i32, i32, f32,
-                                                                 i32, vp, vp, i32, vp, vp, vp, vp]
+                                                                 i32, vp, vp, i32, vp, vp, vp, vp, vp]
+        L.pda_workspace_ints.argtypes = [i32, i32]
+        L.paged_decode_step.argtypes = [vp, vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
+                                        i32, vp, vp, vp, i32, vp, vp, vp]
         L.pda_debug_e4m3_decode.argtypes = [vp, vp]
         L.paged_decode_attention_static.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32,
                                                     f32, i32, i32, vp, vp, vp]
@@ -144,11 +148,42 @@ def paged_decode_reduce(part_o, part_lse, seq_lens, chunk_tokens, out=None, stre
     return out
 
 
+def workspace_ints(batch: int, num_kv_heads: int) -> int:
+    return int(lib().pda_workspace_ints(batch, num_kv_heads))
+
+
+def new_workspace(batch: int, num_kv_heads: int, device="cuda") -> torch.Tensor:
+    """Zeroed int32 workspace for ``paged_decode_step`` (zero it once; calls leave it zeroed)."""
+    return torch.zeros(workspace_ints(batch, num_kv_heads), dtype=torch.int32, device=device)
+
+
+def paged_decode_step(q, k_new, v_new, k_cache, v_cache, block_table, seq_lens, scale,
+                      chunk_tokens=0, out=None, part_o=None, part_lse=None, workspace=None,
+                      k_scale=None, v_scale=None, status=None, stream=None):
+    """Fused append + attention (+ reduce) in one launch; fills and returns ``out``."""
+    desc = cache_desc(k_cache)
+    assert q.is_contiguous() and q.dtype == torch.bfloat16 and block_table.stride(1) == 1
+    B, Hq, D = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    mc = 0
+    if chunk_tokens:
+        mc = part_o.shape[2]
+        assert tuple(part_o.shape) == (B, Hq, mc, D) and tuple(part_lse.shape) == (B, Hq, mc)
+    rc = lib().paged_decode_step(
+        _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), C.byref(desc),
+        _ptr(k_scale), _ptr(v_scale), _ptr(block_table), block_table.stride(0), _ptr(seq_lens),
+        B, Hq, float(scale), chunk_tokens, _ptr(out), _ptr(part_o), _ptr(part_lse), mc,
+        _ptr(workspace), _ptr(status), _stream(stream))
+    _check(rc, "paged_decode_step")
+    return out
+
+
 def paged_decode_step_host(q_host, k_new_host, v_new_host, block_table_host, seq_lens_host,
                            q_dev, k_new_dev, v_new_dev, block_table_dev, seq_lens_dev,
                            k_cache, v_cache, scale, chunk_tokens, part_o, part_lse,
-                           out_dev, out_host, status=None, stream=None):
-    """kv_append + attention (+ reduce) from pinned host inputs to a host output."""
+                           out_dev, out_host, workspace=None, status=None, stream=None):
+    """Fused decode step from pinned host inputs to a host output."""
     desc = cache_desc(k_cache)
     B, Hq, _ = q_host.shape
     mc = 0 if part_o is None else part_o.shape[2]
@@ -157,7 +192,8 @@ def paged_decode_step_host(q_host, k_new_host, v_new_host, block_table_host, seq
         _ptr(seq_lens_host), _ptr(q_dev), _ptr(k_new_dev), _ptr(v_new_dev), _ptr(block_table_dev),
         _ptr(seq_lens_dev), _ptr(k_cache), _ptr(v_cache), C.byref(desc),
         block_table_host.stride(0), B, Hq, float(scale), chunk_tokens, _ptr(part_o),
-        _ptr(part_lse), mc, _ptr(out_dev), _ptr(out_host), _ptr(status), _stream(stream))
+        _ptr(part_lse), mc, _ptr(workspace), _ptr(out_dev), _ptr(out_host), _ptr(status),
+        _stream(stream))
     _check(rc, "paged_decode_step_host")
     return out_host
 

@@ -147,6 +147,54 @@ int paged_decode_attention(const void* q, const void* k_cache, const void* v_cac
   return static_cast<int>(pda::launch_attention_generic(p, s));
 }
 
+int pda_workspace_ints(int32_t batch, int32_t num_kv_heads) {
+  if (batch < 0 || num_kv_heads <= 0) return PDA_ERR_INVALID_ARG;
+  const int64_t n = 2 + static_cast<int64_t>(batch) * num_kv_heads;
+  return n > INT32_MAX ? PDA_ERR_TOO_LARGE : static_cast<int>(n);
+}
+
+int paged_decode_step(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                      void* v_cache, const pda_cache_desc* desc, const float* k_scale,
+                      const float* v_scale, const int32_t* block_table,
+                      int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+                      int32_t num_q_heads, float scale, int32_t chunk_tokens, void* out,
+                      float* part_o, float* part_lse, int32_t max_chunks, int32_t* workspace,
+                      int32_t* status, pda_stream_t stream) {
+  AttnParams p;
+  if (!out && batch > 0) return PDA_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return PDA_ERR_INVALID_ARG;
+  if (int rc = check_attention(q, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                               block_table_stride, seq_lens, batch, num_q_heads, chunk_tokens,
+                               out, part_o, part_lse, max_chunks, &p))
+    return rc;
+  if (k_new && p.geom.dtype != PDA_BF16) return PDA_ERR_UNSUPPORTED;
+  if (k_new && (!aligned16(k_new) || !aligned16(v_new))) return PDA_ERR_MISALIGNED;
+  if (batch == 0) return PDA_OK;
+  p.status = status;
+  p.scale = scale;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  const bool can_fuse = pda::attention_tma_supports(p) && (chunk_tokens == 0 || workspace);
+  if (can_fuse) {
+    pda::StepParams sp{p, k_new, v_new, k_cache, v_cache, workspace, 1};
+    return static_cast<int>(pda::launch_step_tma(sp, static_cast<cudaStream_t>(stream)));
+  }
+  // shapes outside the fused kernel: the same step as separate launches
+  if (k_new) {
+    if (int rc = kv_append(k_new, v_new, k_cache, v_cache, desc, block_table, block_table_stride,
+                           seq_lens, batch, status, stream))
+      return rc;
+  }
+  if (int rc = paged_decode_attention(q, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                                      block_table_stride, seq_lens, batch, num_q_heads, scale,
+                                      chunk_tokens, out, part_o, part_lse, max_chunks, 0u, status,
+                                      stream))
+    return rc;
+  if (chunk_tokens > 0)
+    return paged_decode_reduce(part_o, part_lse, seq_lens, batch, num_q_heads, p.geom.head_dim,
+                               chunk_tokens, max_chunks, out, stream);
+  return PDA_OK;
+}
+
 int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
                         int32_t batch, int32_t num_q_heads, int32_t head_dim,
                         int32_t chunk_tokens, int32_t max_chunks, void* out,
@@ -169,8 +217,8 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
                            void* k_cache, void* v_cache, const pda_cache_desc* desc,
                            int32_t block_table_stride, int32_t batch, int32_t num_q_heads,
                            float scale, int32_t chunk_tokens, float* part_o, float* part_lse,
-                           int32_t max_chunks, void* out_dev, void* out_host, int32_t* status,
-                           pda_stream_t stream) {
+                           int32_t max_chunks, int32_t* workspace, void* out_dev, void* out_host,
+                           int32_t* status, pda_stream_t stream) {
   AttnParams p;
   if (!out_dev || !out_host) return PDA_ERR_INVALID_ARG;
   if (int rc = check_attention(q_dev, k_cache, v_cache, desc, nullptr, nullptr, block_table_dev,
@@ -197,19 +245,11 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
   if ((e = cudaMemcpyAsync(seq_lens_dev, seq_lens_host, static_cast<size_t>(batch) * 4,
                            cudaMemcpyHostToDevice, s)))
     return e;
-  if (int rc = kv_append(k_new_dev, v_new_dev, k_cache, v_cache, desc, block_table_dev,
-                         block_table_stride, seq_lens_dev, batch, status, stream))
+  if (int rc = paged_decode_step(q_dev, k_new_dev, v_new_dev, k_cache, v_cache, desc, nullptr, nullptr,
+                                 block_table_dev, block_table_stride, seq_lens_dev, batch,
+                                 num_q_heads, scale, chunk_tokens, out_dev, part_o, part_lse,
+                                 max_chunks, workspace, status, stream))
     return rc;
-  if (int rc = paged_decode_attention(q_dev, k_cache, v_cache, desc, nullptr, nullptr,
-                                      block_table_dev, block_table_stride, seq_lens_dev, batch,
-                                      num_q_heads, scale, chunk_tokens, out_dev, part_o,
-                                      part_lse, max_chunks, 0u, status, stream))
-    return rc;
-  if (chunk_tokens > 0) {
-    if (int rc = paged_decode_reduce(part_o, part_lse, seq_lens_dev, batch, num_q_heads,
-                                     p.geom.head_dim, chunk_tokens, max_chunks, out_dev, stream))
-      return rc;
-  }
   if ((e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, s))) return e;
   return PDA_OK;
 }

@@ -22,108 +22,19 @@
 // Every wait on an mbarrier is bounded; on expiry the CTA reports
 // PDA_DEV_TIMEOUT, waits (bounded) for its copies in flight and zero-fills its
 // output. TMA copies never use multicast.
-#include <cuda.h>
-#include <cuda_fp16.h>
-
 #include "common.cuh"
+#include "tma_ptx.cuh"
 
 namespace pda {
 
 namespace {
 
-constexpr int kWarps = 4;
-constexpr uint32_t kSpinLimit = 1u << 22;
-
-// ---- PTX wrappers ------------------------------------------------------------------------
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: false if the phase did not complete within kSpinLimit polls.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void fence_proxy_async() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void fence_mbar_init() {
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                            int c0, int c1, int c2, int c3, int c4) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-      : "memory");
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-template <bool kF16>
-__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  if (kF16) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-  } else {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-  }
-}
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
-  uint32_t d;
-  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
-  return d;
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// (lo, hi) fp32 -> packed 16-bit pair, lo in bits 0..15
-template <bool kF16>
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  uint32_t r;
-  if (kF16) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-// two e4m3 bytes (bits 0..15 of x) -> f16x2
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
-  uint32_t r;
-  asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, t;\n\t}" : "=r"(r) : "r"(x));
-  return r;
-}
 
 // ---- kernel ------------------------------------------------------------------------------
 
-template <int D, bool kFp8, int kStages>
+constexpr int kMaxLptBatch = 256;  // above this the O(batch^2 / threads) ranking costs more than it saves
+
+template <int D, bool kFp8, int kStages, int kWarps>
 struct Cfg {
   static constexpr int kElem = kFp8 ? 1 : 2;
   static constexpr int kRowBytes = D * kElem;            // one token row
@@ -138,42 +49,63 @@ struct Cfg {
   static_assert(kMergeBytes <= kWarpRing, "merge buffer reuses the warp's ring");
 };
 
-// Byte offset of 16-byte chunk `chunk` of row `r` inside a tile stored as kSub
-// sub-tiles of [16 rows][128 B] with the 128-byte TMA swizzle.
-__device__ __forceinline__ uint32_t tile_off(int r, int chunk) {
-  return static_cast<uint32_t>((chunk >> 3) * (kPageSize * 128) + r * 128 + (((chunk & 7) ^ (r & 7)) << 4));
-}
-
-template <int D, bool kFp8, int kStages>
+template <int D, bool kFp8, int kStages, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
 attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
-                     const __grid_constant__ CUtensorMap v_map, AttnParams p) {
-  using C = Cfg<D, kFp8, kStages>;
+                     const __grid_constant__ CUtensorMap v_map, StepParams sp) {
+  using C = Cfg<D, kFp8, kStages, kWarps>;
+  const AttnParams& p = sp.a;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kWarps * C::kWarpRing);
-  int* cta_err = reinterpret_cast<int*>(bars + kWarps * kStages);
+  int* cta_err = reinterpret_cast<int*>(bars + kWarps * kStages);  // [0] error code, [1] "last chunk of the unit"
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int gid = lane >> 2, tq = lane & 3;
-  const int c = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int c = blockIdx.x, g = blockIdx.y;
+  int b = blockIdx.z;
+  if (p.chunk_tokens == 0 && p.batch <= kMaxLptBatch && p.batch > 1) {
+    // unsplit units differ in length by the spread of seq_lens: serve the longest first. The CTA
+    // with blockIdx.z = r takes the r-th longest sequence (ties by index), so long units start
+    // early and short ones fill the tail. (Split units are bounded by chunk_tokens already.)
+    int* lens = reinterpret_cast<int*>(smem);
+    for (int j = tid; j < p.batch; j += kWarps * 32) lens[j] = max(p.seq_lens[j], 0);
+    __syncthreads();
+    for (int j = tid; j < p.batch; j += kWarps * 32) {
+      const int Lj = lens[j];
+      int rank = 0;
+      for (int i = 0; i < p.batch; ++i) rank += (lens[i] > Lj) || (lens[i] == Lj && i < j);
+      if (rank == static_cast<int>(blockIdx.z)) cta_err[2] = j;
+    }
+    __syncthreads();
+    b = cta_err[2];
+    __syncthreads();  // lens aliases the ring: done with it before any copy lands
+  }
   const int G = p.group;
   const bool split = p.chunk_tokens > 0;
   const int64_t row0 = static_cast<int64_t>(b) * p.num_q_heads + static_cast<int64_t>(g) * G;
 
+  // fused step: this launch also writes `out` (merging split-KV partials through the
+  // workspace's per-unit chunk counters) and applies the append
+  const bool fuse = sp.fuse_reduce != 0;
   const int L = max(p.seq_lens[b], 0);
   int t0 = 0, t1 = L;
   if (split) {
     t0 = c * p.chunk_tokens;
-    if (t0 >= L) return;
+    if (t0 >= L) {
+      if (fuse && c == 0)  // empty sequence: its output rows are zero
+        for (int i = tid; i < G * D; i += kWarps * 32) p.out[row0 * D + i] = __float2bfloat16_rn(0.f);
+      return;
+    }
     t1 = min(t0 + p.chunk_tokens, L);
   }
+  const int nch = split ? min((L + p.chunk_tokens - 1) / p.chunk_tokens, p.max_chunks) : 1;
   int err = 0;
   if (static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
       (split && static_cast<int64_t>(L) > static_cast<int64_t>(p.max_chunks) * p.chunk_tokens))
     err = PDA_DEV_BAD_SEQ_LEN;
 
-  if (tid == 0) *cta_err = 0;
+  if (tid == 0) { cta_err[0] = 0; cta_err[1] = 0; }
   const int n_tiles = err ? 0 : (t1 - t0 + kPageSize - 1) / kPageSize;
   const int n_mine = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;  // tiles warp, warp+kWarps, ...
   const int page0 = t0 / kPageSize;
@@ -189,16 +121,16 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
 
   // ---- page ids (and e4m3 scales) for this warp's tiles, 32 ordinals per register block
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
-  bool bad_page = false;
+  bool bad_page = false;  // warp-uniform
   auto load_block = [&](int blk, int& pg, float& ks, float& vs) {
     const int kk = blk * 32 + lane;
     pg = 0; ks = 0.f; vs = 0.f;
     if (kk < n_mine) {
       const int v = table[page0 + warp + kk * kWarps];
-      if (v < 0 || v >= p.geom.num_pages) bad_page = true; else pg = v;
+      pg = (v < 0 || v >= p.geom.num_pages) ? -1 : v;  // -1 marks a bad id; clamped where it is used
       if (kFp8) {
-        ks = p.k_scale[static_cast<int64_t>(pg) * p.geom.num_kv_heads + g];
-        vs = p.v_scale[static_cast<int64_t>(pg) * p.geom.num_kv_heads + g];
+        ks = p.k_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g];
+        vs = p.v_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g];
       }
     }
   };
@@ -206,7 +138,8 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
   load_block(0, pgA, ksA, vsA);
   load_block(1, pgB, ksB, vsB);
 
-  auto issue = [&](int kk, int page) {  // lane 0 only
+  auto issue = [&](int kk, int page_raw) {  // lane 0 only
+    const int page = max(page_raw, 0);
     const int s = kk % kStages;
     const uint32_t bar = bar0 + 8 * s;
     const uint32_t dst = ring + s * C::kStageBytes;
@@ -220,9 +153,11 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     const int n_pre = min(kStages, n_mine);
     for (int kk = 0; kk < n_pre; ++kk) {
       const int page = __shfl_sync(0xffffffffu, pgA, kk);
+      if (page < 0) bad_page = true;
       if (lane == 0) issue(kk, page);
     }
   }
+  const bool append_here = sp.k_new != nullptr && !err && c == nch - 1;  // L > 0 here
 
   // ---- Q^T fragments (B operand of S^T = K.Q^T): column n = gid is head gid of the group
   uint32_t qf[C::kKSteps][2];
@@ -275,6 +210,25 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       vsc = __shfl_sync(0xffffffffu, vsA, kk & 31);
     }
 
+    if (!kFp8 && append_here && warp + kk * kWarps == n_tiles - 1) {
+      // fused append: the new token's K/V rows go into the landed tile and into the cache
+      const int slot = (L - 1) % kPageSize;
+      const int page = __shfl_sync(0xffffffffu, pgA, kk & 31);
+      if (lane < C::kRowBytes / 16 && page >= 0) {
+        const int64_t src = (static_cast<int64_t>(b) * p.geom.num_kv_heads + g) * D + lane * 8;
+        const uint4 kv = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(sp.k_new) + src);
+        const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(sp.v_new) + src);
+        const int64_t dst = page * p.geom.page_stride + g * p.geom.head_stride +
+                            slot * p.geom.slot_stride + lane * 8;
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(sp.k_cache_w) + dst) = kv;
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(sp.v_cache_w) + dst) = vv;
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(kt + tile_off(slot, lane)),
+                     "r"(kv.x), "r"(kv.y), "r"(kv.z), "r"(kv.w));
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(vt + tile_off(slot, lane)),
+                     "r"(vv.x), "r"(vv.y), "r"(vv.z), "r"(vv.w));
+      }
+      __syncwarp();
+    }
     if (n_valid < kPageSize) {
       // rows past the sequence end may hold anything: clear them in V (K is masked by select)
       const int n_chunks = C::kRowBytes / 16;
@@ -373,6 +327,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       // kn lies in the consumer's block or the one after it
       const bool in_a = (kn >> 5) == ((kk + 1) >> 5);
       const int page = __shfl_sync(0xffffffffu, in_a ? pgA : pgB, kn & 31);
+      if (page < 0) bad_page = true;
       if (lane == 0) {
         fence_proxy_async();
         issue(kn, page);
@@ -386,7 +341,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       mbar_wait_bounded(bar0 + 8 * (j % kStages), (j / kStages) & 1);
     if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   }
-  if (__any_sync(0xffffffffu, bad_page) && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
+  if (bad_page && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
 
   // ---- publish this warp's state into its own (drained) ring
 #pragma unroll
@@ -442,7 +397,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     }
     const bool live = !dev_err && lsum > 0.f;
     const float val = live ? acc / lsum : 0.f;
-    if (split) {
+    if (split && !(fuse && nch == 1)) {
       const int64_t pr = (row0 + h) * p.max_chunks + c;
       p.part_o[pr * D + d] = val;
       if (d == 0) p.part_lse[pr] = live ? (M + __log2f(lsum)) * kLn2 : -INFINITY;
@@ -450,15 +405,71 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       p.out[(row0 + h) * D + d] = __float2bfloat16_rn(val);
     }
   }
+
+  if (fuse && split && nch > 1) {
+    // ---- fused reduce: publish this chunk, count it in; the unit's last chunk merges them all.
+    // No CTA waits for another one: whoever arrives last finds every partial already visible.
+    int* counter = sp.workspace + 2 + b * p.geom.num_kv_heads + g;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) cta_err[1] = (atomicAdd(counter, 1) == nch - 1) ? 1 : 0;
+    __syncthreads();
+    if (cta_err[1]) {
+      __threadfence();
+      for (int idx = tid; idx < G * D; idx += kWarps * 32) {
+        const int h = idx / D, d = idx % D;
+        const int64_t row = row0 + h;
+        const float* lse = p.part_lse + row * p.max_chunks;
+        float M = -INFINITY;
+        for (int cc = 0; cc < nch; ++cc) M = fmaxf(M, __ldcg(lse + cc));
+        float acc = 0.f, W = 0.f;
+        if (M > -INFINITY) {
+          const float* po = p.part_o + row * p.max_chunks * D + d;
+          for (int cc = 0; cc < nch; ++cc) {
+            const float w = __expf(__ldcg(lse + cc) - M);
+            W += w;
+            acc = fmaf(w, __ldcg(po + static_cast<int64_t>(cc) * D), acc);
+          }
+          acc /= W;
+        }
+        p.out[row * D + d] = __float2bfloat16_rn(acc);
+      }
+      if (tid == 0) *counter = 0;  // leave the workspace clean for the next call
+    }
+  }
 }
 
 // ---- host side ---------------------------------------------------------------------------
 
+template <int D, bool kFp8, int kStages, int kWarps>
+cudaError_t launch(const StepParams& sp, cudaStream_t stream) {
+  using C = Cfg<D, kFp8, kStages, kWarps>;
+  const AttnParams& p = sp.a;
+  alignas(64) CUtensorMap k_map, v_map;
+  const int eb = p.geom.dtype == PDA_BF16 ? 2 : 1;
+  if (!make_cache_tensor_map(&k_map, p.k_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
+                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, eb) ||
+      !make_cache_tensor_map(&v_map, p.v_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
+                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, eb))
+    return cudaErrorNotSupported;
+  auto kern = attention_tma_kernel<D, kFp8, kStages, kWarps>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks) : 1u;
+  dim3 grid(chunks, p.geom.num_kv_heads, p.batch);
+  kern<<<grid, kWarps * 32, C::kSmemBytes, stream>>>(k_map, v_map, sp);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+namespace {
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                               CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                               CUtensorMapFloatOOBfill);
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no libcuda link).
 EncodeFn encode_fn() {
   static EncodeFn fn = [] {
     void* sym = nullptr;
@@ -470,19 +481,20 @@ EncodeFn encode_fn() {
   }();
   return fn;
 }
+}  // namespace
 
-// 5-D view of a cache: (byte-lane within a 128-byte line, slot, line of the row, head, page).
-bool make_map(CUtensorMap* map, const void* base, const CacheGeom& g) {
+bool make_cache_tensor_map(CUtensorMap* map, const void* base, int64_t page_stride,
+                           int64_t head_stride, int64_t slot_stride, int num_pages,
+                           int num_kv_heads, int head_dim, int eb) {
   EncodeFn enc = encode_fn();
   if (!enc) return false;
-  const int eb = g.dtype == PDA_BF16 ? 2 : 1;
   const cuuint64_t line_elems = 128 / eb;
-  const cuuint64_t lines = static_cast<cuuint64_t>(g.head_dim) * eb / 128;
+  const cuuint64_t lines = static_cast<cuuint64_t>(head_dim) * eb / 128;
   cuuint64_t dims[5] = {line_elems, static_cast<cuuint64_t>(kPageSize), lines,
-                        static_cast<cuuint64_t>(g.num_kv_heads), static_cast<cuuint64_t>(g.num_pages)};
-  cuuint64_t strides[4] = {static_cast<cuuint64_t>(g.slot_stride) * eb, 128,
-                           static_cast<cuuint64_t>(g.head_stride) * eb,
-                           static_cast<cuuint64_t>(g.page_stride) * eb};
+                        static_cast<cuuint64_t>(num_kv_heads), static_cast<cuuint64_t>(num_pages)};
+  cuuint64_t strides[4] = {static_cast<cuuint64_t>(slot_stride) * eb, 128,
+                           static_cast<cuuint64_t>(head_stride) * eb,
+                           static_cast<cuuint64_t>(page_stride) * eb};
   cuuint32_t box[5] = {static_cast<cuuint32_t>(line_elems), kPageSize, static_cast<cuuint32_t>(lines), 1, 1};
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   const CUresult r = enc(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 5,
@@ -492,23 +504,6 @@ bool make_map(CUtensorMap* map, const void* base, const CacheGeom& g) {
   return r == CUDA_SUCCESS;
 }
 
-template <int D, bool kFp8, int kStages>
-cudaError_t launch(const AttnParams& p, cudaStream_t stream) {
-  using C = Cfg<D, kFp8, kStages>;
-  alignas(64) CUtensorMap k_map, v_map;
-  if (!make_map(&k_map, p.k_cache, p.geom) || !make_map(&v_map, p.v_cache, p.geom))
-    return cudaErrorNotSupported;
-  auto kern = attention_tma_kernel<D, kFp8, kStages>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-  if (e != cudaSuccess) return e;
-  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks) : 1u;
-  dim3 grid(chunks, p.geom.num_kv_heads, p.batch);
-  kern<<<grid, kWarps * 32, C::kSmemBytes, stream>>>(k_map, v_map, p);
-  return cudaGetLastError();
-}
-
-}  // namespace
-
 bool attention_tma_supports(const AttnParams& p) {
   if (p.group < 1 || p.group > 8) return false;
   if (p.geom.num_kv_heads > 65535) return false;
@@ -517,12 +512,18 @@ bool attention_tma_supports(const AttnParams& p) {
   return p.geom.head_dim == 128;
 }
 
-cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream) {
+cudaError_t launch_step_tma(const StepParams& sp, cudaStream_t stream) {
+  const AttnParams& p = sp.a;
   if (p.geom.dtype == PDA_BF16) {
-    if (p.geom.head_dim == 128) return launch<128, false, 3>(p, stream);
-    return launch<64, false, 3>(p, stream);
+    if (p.geom.head_dim == 128) return launch<128, false, 3, 4>(sp, stream);
+    return launch<64, false, 3, 4>(sp, stream);
   }
-  return launch<128, true, 3>(p, stream);
+  return launch<128, true, 3, 4>(sp, stream);
+}
+
+cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream) {
+  const StepParams sp{p, nullptr, nullptr, nullptr, nullptr, nullptr, 0};
+  return launch_step_tma(sp, stream);
 }
 
 }  // namespace pda

@@ -35,6 +35,18 @@ struct AttnParams {
   float scale;
 };
 
+// Fused decode step (attention_tma.cu): attention parameters plus the
+// optional append inputs, the optional workspace and the reduce switch.
+struct StepParams {
+  AttnParams a;
+  const void* k_new;   // [B,Hkv,D] bf16 or nullptr (no append)
+  const void* v_new;
+  void* k_cache_w;     // writable aliases of a.k_cache / a.v_cache (append target)
+  void* v_cache_w;
+  int32_t* workspace;  // per-(sequence, kv head) chunk counters at [2 ..); nullptr when nothing is counted
+  int32_t fuse_reduce; // 1: the launch writes `out` itself (needs workspace when split)
+};
+
 __device__ __forceinline__ void report(int32_t* status, int code) {
   if (status != nullptr) atomicMax(status, code);
 }
@@ -69,6 +81,8 @@ cudaError_t launch_attention_generic(const AttnParams& p, cudaStream_t stream);
 // Returns cudaErrorNotSupported when the shape is outside the fast kernel's set.
 cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream);
 bool attention_tma_supports(const AttnParams& p);
+// Fused step on the same kernel: optional append, optional in-kernel reduce (sp.fuse_reduce).
+cudaError_t launch_step_tma(const StepParams& sp, cudaStream_t stream);
 cudaError_t launch_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
                           int32_t batch, int32_t num_q_heads, int32_t head_dim,
                           int32_t chunk_tokens, int32_t max_chunks, __nv_bfloat16* out,

@@ -1,7 +1,9 @@
 """GPU parity at the full sizes of the five named workloads, in the launch
-configuration bench.py times (same chunk choices), against the full oracle."""
+configuration bench.py times (the fused paged_decode_step with the same chunk
+choices) and through the three separate calls, against the full oracle."""
 import numpy as np
 import pytest
+import torch
 
 from paper_2605_06068_b200 import binding as pda
 from paper_2605_06068_b200 import workloads as W
@@ -10,27 +12,46 @@ from util import DeviceWorkload, assert_close, bf16_to_bits, bf16_to_f64, host_a
 
 pytestmark = pytest.mark.gpu
 
-# (workload, chunk_tokens used by bench.py; 0 = unsplit as well)
-CASES = [("llama8b", 512), ("longctx", 2048), ("chat70b", 512), ("prefix_fp8", 512)]
+# (workload, chunk_tokens bench.py uses for the fused step, chunk_tokens for the separate calls)
+CASES = [("llama8b", 0, 512), ("longctx", 2048, 2048), ("chat70b", 0, 512), ("prefix_fp8", 0, 512)]
 
 
-@pytest.mark.parametrize("name,chunk", CASES)
-def test_full_size_config(oracle, name, chunk):
+@pytest.mark.parametrize("name,chunk,chunk_sep", CASES)
+def test_full_size_config(oracle, name, chunk, chunk_sep):
     w = W.WORKLOADS[name]()
     if w.chunk_tokens:
         assert chunk == w.chunk_tokens
-    dw = DeviceWorkload(w)
     k, v = host_appended(oracle, w)
+    ref = oracle_out(oracle, w, k, v)
+    ref_rms = np.sqrt((ref ** 2).mean())
+
+    # ---- the fused step, as timed by bench.py
+    dw = DeviceWorkload(w)
+    ws = pda.new_workspace(w.batch, w.num_kv_heads)
+    po = pl = None
+    if chunk:
+        mc = pda.max_chunks(int(w.seq_lens.max()), chunk)
+        po = torch.empty((w.batch, w.num_q_heads, mc, w.head_dim), dtype=torch.float32, device="cuda")
+        pl = torch.empty((w.batch, w.num_q_heads, mc), dtype=torch.float32, device="cuda")
+    out = pda.paged_decode_step(dw.q, dw.k_new, dw.v_new, dw.k_cache, dw.v_cache, dw.block_table,
+                                dw.seq_lens, float(w.scale), chunk_tokens=chunk, part_o=po, part_lse=pl,
+                                workspace=ws, k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+    torch.cuda.synchronize()
+    if w.kv_dtype == "bf16":
+        assert (bf16_to_bits(dw.k_cache) == k).all() and (bf16_to_bits(dw.v_cache) == v).all()
+    got = bf16_to_f64(out)
+    worst, nerr = assert_close(got, ref, w.kv_dtype, what=f"{name} fused chunk {chunk}")
+    print(f"{name}: fused chunk {chunk}: max err/tol {worst:.3f}, max err/rms {nerr:.3e}")
+    assert (ws == 0).all() and int(dw.status.item()) == 0
+    # the output is not trivially small: the stated tolerance alone cannot tell at long context
+    assert np.sqrt((got ** 2).mean()) > 0.5 * ref_rms
+
+    # ---- the three separate calls (kv_append, split attention, reduce)
+    dw = DeviceWorkload(w)
     if w.kv_dtype == "bf16":
         dw.append()
         assert (bf16_to_bits(dw.k_cache) == k).all() and (bf16_to_bits(dw.v_cache) == v).all()
-    ref = oracle_out(oracle, w, k, v)
-    out = bf16_to_f64(dw.attend(chunk_tokens=chunk))
-    worst, nerr = assert_close(out, ref, w.kv_dtype, what=f"{name} chunk {chunk}")
-    print(f"{name}: chunk {chunk}: max err/tol {worst:.3f}, max err/rms {nerr:.3e}")
-    if name != "longctx":   # one unit per (sequence, kv head) would serialise 131k tokens
-        out_u = bf16_to_f64(dw.attend())
-        assert_close(out_u, ref, w.kv_dtype, what=f"{name} unsplit")
+    got = bf16_to_f64(dw.attend(chunk_tokens=chunk_sep))
+    worst, nerr = assert_close(got, ref, w.kv_dtype, what=f"{name} separate chunk {chunk_sep}")
+    print(f"{name}: separate chunk {chunk_sep}: max err/tol {worst:.3f}, max err/rms {nerr:.3e}")
     assert int(dw.status.item()) == 0
-    # the output is not trivially small: the stated tolerance alone cannot tell at long context
-    assert np.sqrt((out ** 2).mean()) > 0.5 * np.sqrt((ref ** 2).mean())

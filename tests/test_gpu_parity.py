@@ -14,7 +14,7 @@ from util import (DeviceWorkload, assert_close, bf16_tensor, bf16_to_bits, bf16_
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [pytest.param(0, id="fast"), pytest.param(pda.PDA_FLAG_FORCE_GENERIC, id="generic")]
+PATHS = [pytest.param(0, id="tma"), pytest.param(pda.PDA_FLAG_FORCE_GENERIC, id="generic")]
 
 
 def status_of(dw):
@@ -297,6 +297,90 @@ def test_bad_block_table_sets_status_and_zero_fills(oracle, flags):
     assert (out[2] == 0).all()
 
 
+# ---- the fused step (append + attention + reduce in one launch) -----------------------------
+
+STEP_CASES = [
+    ([17, 33, 64, 100], 8, 2, 64),
+    ([1, 16, 17, 129, 640, 2049, 0, 5], 32, 8, 128),
+    ([5, 48, 300, 777, 1], 64, 8, 128),
+    ([3, 100, 513], 8, 8, 128),
+]
+
+
+@pytest.mark.parametrize("case", STEP_CASES, ids=lambda c: f"Hq{c[1]}kv{c[2]}D{c[3]}")
+def test_fused_step_matches_oracle_and_appends_bit_exactly(oracle, case):
+    lens, Hq, Hkv, D = case
+    w = W.make_workload("step", lens, Hq, Hkv, D, seed=123)
+    k_ref, v_ref = host_appended(oracle, w)
+    ref = oracle_out(oracle, w, k_ref, v_ref)
+    ws = pda.new_workspace(w.batch, Hkv)
+    for chunk in (0, 64, 512):
+        dw = DeviceWorkload(w)
+        po = pl = None
+        if chunk:
+            mc = pda.max_chunks(max(lens), chunk)
+            po = torch.full((w.batch, Hq, mc, D), float("nan"), dtype=torch.float32, device="cuda")
+            pl = torch.full((w.batch, Hq, mc), float("nan"), dtype=torch.float32, device="cuda")
+        out = torch.full_like(dw.q, float("nan"))
+        for rep in range(2):   # the second call re-appends the same rows and reuses the workspace
+            pda.paged_decode_step(dw.q, dw.k_new, dw.v_new, dw.k_cache, dw.v_cache, dw.block_table,
+                                  dw.seq_lens, float(w.scale), chunk_tokens=chunk, out=out,
+                                  part_o=po, part_lse=pl, workspace=ws, status=dw.status)
+            torch.cuda.synchronize()
+            assert (bf16_to_bits(dw.k_cache) == k_ref).all() and (bf16_to_bits(dw.v_cache) == v_ref).all()
+            assert_close(bf16_to_f64(out), ref, what=f"fused step chunk {chunk} rep {rep}")
+            assert (ws == 0).all(), "the workspace must be left zeroed"
+            assert status_of(dw) == 0
+        # same bits as the three separate calls
+        dw3 = DeviceWorkload(w)
+        dw3.append()
+        assert (bf16_to_bits(dw3.attend(chunk_tokens=chunk)) == bf16_to_bits(out)).all()
+
+
+def test_fused_step_fp8_and_no_append(oracle):
+    w = W.prefix_fp8(seed=46, batch=6)
+    dw = DeviceWorkload(w)
+    ref = oracle_out(oracle, w)
+    ws = pda.new_workspace(w.batch, w.num_kv_heads)
+    mc = pda.max_chunks(int(w.seq_lens.max()), 256)
+    po = torch.empty((w.batch, 32, mc, 128), dtype=torch.float32, device="cuda")
+    pl = torch.empty((w.batch, 32, mc), dtype=torch.float32, device="cuda")
+    out = pda.paged_decode_step(dw.q, None, None, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                float(w.scale), chunk_tokens=256, part_o=po, part_lse=pl, workspace=ws,
+                                k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+    assert_close(bf16_to_f64(out), ref, "e4m3", what="fused fp8 step")
+    assert (ws == 0).all() and status_of(dw) == 0
+    # without a workspace the split step falls back to separate launches, same result
+    out2 = pda.paged_decode_step(dw.q, None, None, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                 float(w.scale), chunk_tokens=256, part_o=po, part_lse=pl,
+                                 k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+    assert (bf16_to_bits(out2) == bf16_to_bits(out)).all()
+
+
+def test_fused_step_bad_inputs(oracle):
+    w = W.make_workload("bad", [100, 200, 300], 8, 2, 64, seed=9)
+    dw = DeviceWorkload(w)
+    ws = pda.new_workspace(3, 2)
+    mc = 8
+    po = torch.empty((3, 8, mc, 64), dtype=torch.float32, device="cuda")
+    pl = torch.empty((3, 8, mc), dtype=torch.float32, device="cuda")
+    good = bf16_to_bits(pda.paged_decode_step(dw.q, dw.k_new, dw.v_new, dw.k_cache, dw.v_cache, dw.block_table,
+                                              dw.seq_lens, float(w.scale), chunk_tokens=64, part_o=po,
+                                              part_lse=pl, workspace=ws, status=dw.status)).copy()
+    k_before = bf16_to_bits(dw.k_cache).copy()
+    dw.block_table[0, 3] = -1
+    dw.block_table[1, 12] = w.num_pages      # the page row 1 appends into (L=200 -> logical page 12)
+    out = bf16_to_bits(pda.paged_decode_step(dw.q, dw.k_new, dw.v_new, dw.k_cache, dw.v_cache, dw.block_table,
+                                             dw.seq_lens, float(w.scale), chunk_tokens=64, part_o=po,
+                                             part_lse=pl, workspace=ws, status=dw.status))
+    torch.cuda.synchronize()
+    assert status_of(dw) == 1 and (ws == 0).all()
+    assert (out[2] == good[2]).all()
+    # rows with a bad page: only the chunks that hit it are dropped, nothing is written out of range
+    assert np.isfinite(bf16_to_f64(torch.from_numpy(out.view(np.int16)).view(torch.bfloat16))).all()
+    assert (bf16_to_bits(dw.k_cache) == k_before).all()
+
+
 # ---- reduce on synthetic partials ----------------------------------------------------------
 
 def test_reduce_alone(oracle):
@@ -338,7 +422,8 @@ def test_step_host_matches_device_calls(oracle):
         out_host = torch.zeros(w.q.shape, dtype=torch.int16).pin_memory()
         pda.paged_decode_step_host(hq.view(torch.bfloat16), hk, hv, hbt, hsl, dq, dk, dv, dbt, dsl,
                                    dw.k_cache, dw.v_cache, float(w.scale), chunk, po, pl,
-                                   out_dev, out_host, status=dw.status)
+                                   out_dev, out_host, workspace=pda.new_workspace(w.batch, 8),
+                                   status=dw.status)
         torch.cuda.synchronize()
         got = W.bf16_bits_to_f32(out_host.numpy().view(np.uint16)).astype(np.float64)
         assert_close(got, ref, what=f"step_host chunk {chunk}")
