@@ -256,6 +256,27 @@ def run_gpu(args):
     if int(status.item()) != 0:
         raise RuntimeError(f"device status {int(status.item())}: {pda.status_string(int(status.item()))}")
 
+    # ---- the same step captured once in a CUDA graph and replayed (no host launch work) --------
+    ms_graph = 0.0
+    if not args.no_graph:
+        cap = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        cap.wait_stream(stream)
+        with torch.cuda.stream(cap):
+            with torch.cuda.graph(graph, stream=cap):
+                step()   # the binding launches on the current stream, which is `cap` here
+        barrier()
+        for _ in range(3):
+            graph.replay()
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        g1.record()
+        barrier()
+        ms_graph = g0.elapsed_time(g1) / args.steps
+
     # ---- end to end from pinned host buffers (bf16 workloads) --------------------------------
     e2e = None
     if k_new is not None:
@@ -286,8 +307,9 @@ def run_gpu(args):
 
     # ---- aggregate over ranks ----------------------------------------------------------------
     from paper_2605_06068_b200.sharding import aggregate
-    (ms_step, ms_attn, ms_e2e), (kv_bytes_all, batch_all) = aggregate(
-        [ms_step, ms_attn, e2e[0] if e2e else 0.0], [float(w.kv_bytes), float(w.batch)], device=dev)
+    (ms_step, ms_attn, ms_e2e, ms_graph), (kv_bytes_all, batch_all) = aggregate(
+        [ms_step, ms_attn, e2e[0] if e2e else 0.0, ms_graph], [float(w.kv_bytes), float(w.batch)],
+        device=dev)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -310,6 +332,9 @@ def run_gpu(args):
             "gpu_launches": launches_per_step * args.steps,
             "clocks": sampler.summary(),
         }
+        if ms_graph > 0:
+            line["cuda_graph_replay"] = {"ms_per_step": ms_graph,
+                                         "value": kv_bytes_all / (ms_graph * 1e-3) / 1e9, "unit": "GB/s"}
         if e2e:
             line["e2e"] = {"value": kv_bytes_all / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s",
                            "ms_per_step": ms_e2e, "h2d_bytes_per_step": e2e[1],
@@ -335,6 +360,7 @@ def main():
     ap.add_argument("--workload", default="llama8b", choices=list(W.WORKLOADS))
     ap.add_argument("--chunk", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
     ap.add_argument("--path", default="fused", choices=["fused", "separate"],
                     help="fused: one paged_decode_step launch; separate: kv_append, attention, reduce")
     ap.add_argument("--kernel", default="tma", choices=["tma", "generic"],

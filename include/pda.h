@@ -179,6 +179,15 @@ int paged_decode_step(const void* q, const void* k_new, const void* v_new, void*
                       float* part_o, float* part_lse, int32_t max_chunks, int32_t* workspace,
                       int32_t* status, pda_stream_t stream);
 
+/* seq_lens[b] += delta for every b, on the device and in stream order. Lets a
+ * whole decode step -- advance the lengths, then paged_decode_step -- be captured
+ * once in a CUDA graph and replayed every token with no host work (CUDA-graph
+ * capture of the step is the most frequent single win the paper reports:
+ * Section 4.2, Scenarios B, C, D and F). Grids never depend on seq_lens, the
+ * caches' addresses are baked into the captured launch, and the block table must
+ * already hold the pages the growing sequences will reach. */
+int pda_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t delta, pda_stream_t stream);
+
 /* One whole decode step driven from HOST buffers (the end-to-end call): copies
  * this step's q, k_new, v_new, seq_lens and block_table from (ideally pinned)
  * host memory into the caller's device staging buffers, runs

@@ -22,7 +22,7 @@ DEV_STATUS = {0: "ok", 1: "bad page id", 2: "seq_len exceeds block table", 3: "c
 EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
            "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
-           "paged_decode_step"]
+           "paged_decode_step", "pda_advance_seq_lens"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
@@ -56,6 +56,7 @@ def lib():
         L.paged_decode_step_host.argtypes = [vp] * 5 + [vp] * 5 + [vp, vp, dp, i32, i32, i32, f32,
                                                                  i32, vp, vp, i32, vp, vp, vp, vp, vp]
         L.pda_workspace_ints.argtypes = [i32, i32]
+        L.pda_advance_seq_lens.argtypes = [vp, i32, i32, vp]
         L.paged_decode_step.argtypes = [vp, vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
                                         i32, vp, vp, vp, i32, vp, vp, vp]
         L.pda_debug_e4m3_decode.argtypes = [vp, vp]
@@ -221,3 +222,9 @@ def paged_decode_attention_static(q, k_cache, v_cache, block_table, seq_lens, sc
         chunk_tokens, max_chunks, _ptr(out), _ptr(status), _stream(stream))
     _check(rc, "paged_decode_attention_static")
     return out
+
+
+def advance_seq_lens(seq_lens, delta=1, stream=None):
+    """``seq_lens += delta`` on the device, in stream order (graph-capturable)."""
+    _check(lib().pda_advance_seq_lens(_ptr(seq_lens), seq_lens.shape[0], int(delta), _stream(stream)),
+           "pda_advance_seq_lens")

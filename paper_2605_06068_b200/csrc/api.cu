@@ -254,6 +254,14 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
   return PDA_OK;
 }
 
+int pda_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t delta, pda_stream_t stream) {
+  if (batch < 0) return PDA_ERR_INVALID_ARG;
+  if (batch == 0) return PDA_OK;
+  if (!seq_lens) return PDA_ERR_INVALID_ARG;
+  return static_cast<int>(pda::launch_advance_seq_lens(seq_lens, batch, delta,
+                                                       static_cast<cudaStream_t>(stream)));
+}
+
 int pda_debug_e4m3_decode(float* out256, pda_stream_t stream) {
   if (!out256) return PDA_ERR_INVALID_ARG;
   return static_cast<int>(pda::launch_e4m3_decode(out256, static_cast<cudaStream_t>(stream)));

@@ -49,4 +49,15 @@ cudaError_t launch_kv_append(const void* k_new, const void* v_new, void* k_cache
   return cudaGetLastError();
 }
 
+__global__ void advance_seq_lens_kernel(int32_t* seq_lens, int32_t batch, int32_t delta) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < batch) seq_lens[b] += delta;
+}
+
+cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t delta, cudaStream_t stream) {
+  if (batch == 0) return cudaSuccess;
+  advance_seq_lens_kernel<<<(batch + 255) / 256, 256, 0, stream>>>(seq_lens, batch, delta);
+  return cudaGetLastError();
+}
+
 }  // namespace pda
