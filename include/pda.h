@@ -142,6 +142,25 @@ int paged_decode_attention(const void* q, const void* k_cache, const void* v_cac
                            int32_t max_chunks, uint32_t flags, int32_t* status,
                            pda_stream_t stream);
 
+/* Sliding-window decode attention: paged_decode_attention restricted, for every
+ * sequence, to its last `window` tokens j in [max(0, L - window), L) (the
+ * sliding-window attention over a paged per-stream cache of the paper's
+ * streaming scenario, Appendix A, Scenario D; the paper gives no formula -- this
+ * is the same softmax over that token range). window == 0 means no window.
+ * Pages wholly before the window are never read, so their block_table entries
+ * may be stale (evicted pages). With chunk_tokens > 0 the chunk grid stays the
+ * one of the full sequence: chunks wholly before the window get o = 0 and
+ * lse = -inf, and paged_decode_reduce merges as usual. Other arguments as in
+ * paged_decode_attention. */
+int paged_window_decode_attention(const void* q, const void* k_cache, const void* v_cache,
+                                  const pda_cache_desc* desc, const float* k_scale,
+                                  const float* v_scale, const int32_t* block_table,
+                                  int32_t block_table_stride, const int32_t* seq_lens,
+                                  int32_t batch, int32_t num_q_heads, float scale, int32_t window,
+                                  int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                                  int32_t max_chunks, uint32_t flags, int32_t* status,
+                                  pda_stream_t stream);
+
 /* Merge of split-KV partials (the reduce step of flash-decoding; exact algebra):
  *     out[b,h,:] = sum_c w_c part_o[b,h,c,:] / sum_c w_c,
  *     w_c = exp(part_lse[b,h,c] - max_c part_lse[b,h,c]),  c < ceil(L_b/chunk_tokens)

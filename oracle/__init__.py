@@ -82,9 +82,10 @@ def kv_append(k_new, v_new, k_cache, v_cache, block_table, seq_lens):
 
 def paged_decode_attention(q, k_cache, v_cache, block_table, seq_lens, scale,
                            k_scale=None, v_scale=None, chunk_tokens=0, max_chunks=0,
-                           n_threads=0):
+                           n_threads=0, window=0):
     """Returns ``(out, lse)`` in float64.
 
+    ``window > 0`` attends only each sequence's last ``window`` tokens.
     Unsplit: ``out [B,Hq,D]``, ``lse [B,Hq]``. Split (``chunk_tokens > 0``):
     ``out [B,Hq,max_chunks,D]`` (NaN where no chunk exists) and
     ``lse [B,Hq,max_chunks]`` (NaN likewise).
@@ -123,7 +124,7 @@ def paged_decode_attention(q, k_cache, v_cache, block_table, seq_lens, scale,
         C.c_int64(ps), C.c_int64(hs), C.c_int64(ss), C.c_int32(P), C.c_int32(Hkv),
         C.c_int32(D), _p(block_table), C.c_int32(block_table.shape[1]), _p(seq_lens),
         C.c_int32(B), C.c_int32(Hq), C.c_float(np.float32(scale)), C.c_int32(chunk_tokens),
-        C.c_int32(max_chunks), _p(out), _p(lse), C.c_int32(n_threads))
+        C.c_int32(max_chunks), C.c_int32(window), _p(out), _p(lse), C.c_int32(n_threads))
     return out, lse
 
 

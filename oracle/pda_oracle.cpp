@@ -183,7 +183,10 @@ void oracle_kv_append(const uint8_t* k_new, const uint8_t* v_new, uint8_t* k_cac
   }
 }
 
-// Attention. chunk_tokens == 0: out is [B,Hq,D], lse is [B,Hq].
+// Attention. window > 0 restricts every sequence to its last `window` tokens
+// (the sliding-window attention of the paper's streaming scenario, Appendix A,
+// Scenario D; the definition is the same softmax over that token range).
+// chunk_tokens == 0: out is [B,Hq,D], lse is [B,Hq].
 // chunk_tokens  > 0: out is [B,Hq,max_chunks,D], lse is [B,Hq,max_chunks];
 // entries for chunks c >= ceil(L_b / chunk_tokens) are left untouched.
 // kv_dtype: 0 = bf16, 1 = e4m3 with k_scale/v_scale [num_pages,Hkv] fp32.
@@ -193,7 +196,7 @@ void oracle_paged_decode_attention(
     int64_t slot_stride, int32_t page_size, int32_t num_kv_heads, int32_t head_dim,
     const int32_t* block_table, int32_t block_table_stride, const int32_t* seq_lens,
     int32_t batch, int32_t num_q_heads, float scale, int32_t chunk_tokens, int32_t max_chunks,
-    double* out, double* lse, int32_t n_threads) {
+    int32_t window, double* out, double* lse, int32_t n_threads) {
   const int G = num_q_heads / num_kv_heads;
   const CacheView K{k_cache, kv_dtype, page_stride, head_stride, slot_stride, k_scale, num_kv_heads};
   const CacheView V{v_cache, kv_dtype, page_stride, head_stride, slot_stride, v_scale, num_kv_heads};
@@ -206,14 +209,17 @@ void oracle_paged_decode_attention(
     const int64_t L = seq_lens[b] > 0 ? seq_lens[b] : 0;
     const uint16_t* q_row = q + row * head_dim;
     const int32_t* table_row = block_table + static_cast<int64_t>(b) * block_table_stride;
+    // sliding window: only the last `window` tokens are attended (window <= 0: all of them)
+    const int64_t lo = (window > 0 && L > window) ? L - window : 0;
     if (chunk_tokens == 0) {
-      attend_range(q_row, K, V, table_row, page_size, head_dim, g, sc, 0, L,
+      attend_range(q_row, K, V, table_row, page_size, head_dim, g, sc, lo, L,
                    out + row * head_dim, lse + row);
     } else {
       const int64_t n_chunks = (L + chunk_tokens - 1) / chunk_tokens;
       for (int64_t c = 0; c < n_chunks; ++c) {
-        const int64_t t0 = c * chunk_tokens;
+        int64_t t0 = c * chunk_tokens;
         const int64_t t1 = (t0 + chunk_tokens < L) ? t0 + chunk_tokens : L;
+        if (t0 < lo) t0 = lo;  // a chunk wholly before the window is an empty range (o = 0, lse = -inf)
         attend_range(q_row, K, V, table_row, page_size, head_dim, g, sc, t0, t1,
                      out + (row * max_chunks + c) * head_dim, lse + row * max_chunks + c);
       }

@@ -22,7 +22,7 @@ DEV_STATUS = {0: "ok", 1: "bad page id", 2: "seq_len exceeds block table", 3: "c
 EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
            "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
-           "paged_decode_step", "pda_advance_seq_lens"]
+           "paged_decode_step", "pda_advance_seq_lens", "paged_window_decode_attention"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
@@ -56,6 +56,8 @@ def lib():
         L.paged_decode_step_host.argtypes = [vp] * 5 + [vp] * 5 + [vp, vp, dp, i32, i32, i32, f32,
                                                                  i32, vp, vp, i32, vp, vp, vp, vp, vp]
         L.pda_workspace_ints.argtypes = [i32, i32]
+        L.paged_window_decode_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
+                                                    i32, i32, vp, vp, vp, i32, u32, vp, vp]
         L.pda_advance_seq_lens.argtypes = [vp, i32, i32, vp]
         L.paged_decode_step.argtypes = [vp, vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
                                         i32, vp, vp, vp, i32, vp, vp, vp]
@@ -136,6 +138,28 @@ def paged_decode_attention(q, k_cache, v_cache, block_table, seq_lens, scale, ch
         chunk_tokens, _ptr(out), _ptr(part_o), _ptr(part_lse), mc, flags, _ptr(status),
         _stream(stream))
     _check(rc, "paged_decode_attention")
+    return out if chunk_tokens == 0 else (part_o, part_lse)
+
+
+def paged_window_decode_attention(q, k_cache, v_cache, block_table, seq_lens, scale, window,
+                                  chunk_tokens=0, out=None, part_o=None, part_lse=None,
+                                  k_scale=None, v_scale=None, flags=0, status=None, stream=None):
+    """``paged_decode_attention`` over each sequence's last ``window`` tokens only."""
+    desc = cache_desc(k_cache)
+    B, Hq, D = q.shape
+    mc = 0
+    if chunk_tokens == 0:
+        if out is None:
+            out = torch.empty_like(q)
+    else:
+        mc = part_o.shape[2]
+        assert tuple(part_o.shape) == (B, Hq, mc, D) and tuple(part_lse.shape) == (B, Hq, mc)
+    rc = lib().paged_window_decode_attention(
+        _ptr(q), _ptr(k_cache), _ptr(v_cache), C.byref(desc), _ptr(k_scale), _ptr(v_scale),
+        _ptr(block_table), block_table.stride(0), _ptr(seq_lens), B, Hq, float(scale), int(window),
+        chunk_tokens, _ptr(out), _ptr(part_o), _ptr(part_lse), mc, flags, _ptr(status),
+        _stream(stream))
+    _check(rc, "paged_window_decode_attention")
     return out if chunk_tokens == 0 else (part_o, part_lse)
 
 

@@ -78,6 +78,9 @@ int check_attention(const void* q, const void* k_cache, const void* v_cache,
   p->chunk_tokens = chunk_tokens;
   p->max_chunks = max_chunks;
   p->scale = 0.f;
+  p->window = 0;
+  p->first_token = 0;
+  p->chunk_slot0 = 0;
   return PDA_OK;
 }
 
@@ -147,6 +150,30 @@ int paged_decode_attention(const void* q, const void* k_cache, const void* v_cac
   return static_cast<int>(pda::launch_attention_generic(p, s));
 }
 
+int paged_window_decode_attention(const void* q, const void* k_cache, const void* v_cache,
+                                  const pda_cache_desc* desc, const float* k_scale,
+                                  const float* v_scale, const int32_t* block_table,
+                                  int32_t block_table_stride, const int32_t* seq_lens,
+                                  int32_t batch, int32_t num_q_heads, float scale, int32_t window,
+                                  int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                                  int32_t max_chunks, uint32_t flags, int32_t* status,
+                                  pda_stream_t stream) {
+  AttnParams p;
+  if (window < 0) return PDA_ERR_INVALID_ARG;
+  if (int rc = check_attention(q, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                               block_table_stride, seq_lens, batch, num_q_heads, chunk_tokens,
+                               out, part_o, part_lse, max_chunks, &p))
+    return rc;
+  if (batch == 0) return PDA_OK;
+  p.status = status;
+  p.scale = scale;
+  p.window = window;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (!(flags & PDA_FLAG_FORCE_GENERIC) && pda::attention_tma_supports(p))
+    return static_cast<int>(pda::launch_attention_tma(p, s));
+  return static_cast<int>(pda::launch_attention_generic(p, s));
+}
+
 int pda_workspace_ints(int32_t batch, int32_t num_kv_heads) {
   if (batch < 0 || num_kv_heads <= 0) return PDA_ERR_INVALID_ARG;
   const int64_t n = 2 + static_cast<int64_t>(batch) * num_kv_heads;
@@ -205,7 +232,7 @@ int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_
   if (batch == 0) return PDA_OK;
   if (!part_o || !part_lse || !seq_lens || !out) return PDA_ERR_INVALID_ARG;
   return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
-                                             head_dim, chunk_tokens, max_chunks,
+                                             head_dim, chunk_tokens, max_chunks, 0, 0,
                                              static_cast<__nv_bfloat16*>(out),
                                              static_cast<cudaStream_t>(stream)));
 }

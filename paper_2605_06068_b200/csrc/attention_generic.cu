@@ -30,15 +30,18 @@ __global__ void __launch_bounds__(32) attention_generic_kernel(AttnParams p) {
   const bool split = p.chunk_tokens > 0;
 
   const int L = max(p.seq_lens[b], 0);
-  int t0 = 0, t1 = L;
+  int t0 = p.first_token, t1 = L;
   if (split) {
-    t0 = c * p.chunk_tokens;
+    t0 = p.first_token + c * p.chunk_tokens;
     if (t0 >= L) return;  // no such chunk
     t1 = min(t0 + p.chunk_tokens, L);
   }
+  // window: tokens before L - window are not attended; the unit may end up empty
+  if (p.window > 0 && L - p.window > t0) t0 = min(L - p.window, t1);
   const bool too_long =
       static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
-      (split && static_cast<int64_t>(L) > static_cast<int64_t>(p.max_chunks) * p.chunk_tokens);
+      (split && static_cast<int64_t>(L - p.first_token) >
+                    static_cast<int64_t>(p.max_chunks - p.chunk_slot0) * p.chunk_tokens);
 
   __shared__ float q_s[256];
   for (int d = lane; d < D; d += 32) q_s[d] = __bfloat162float(p.q[row * D + d]);
@@ -104,8 +107,8 @@ __global__ void __launch_bounds__(32) attention_generic_kernel(AttnParams p) {
   if (failed && lane == 0) report(p.status, too_long ? PDA_DEV_BAD_SEQ_LEN : PDA_DEV_BAD_PAGE);
   const float inv_l = (l > 0.f && !failed) ? 1.f / l : 0.f;
   if (split) {
-    const int64_t pr = row * p.max_chunks + c;
-    if (c >= p.max_chunks) return;
+    const int64_t pr = row * p.max_chunks + p.chunk_slot0 + c;
+    if (p.chunk_slot0 + c >= p.max_chunks) return;
 #pragma unroll
     for (int i = 0; i < kMaxDPerLane; ++i) {
       const int d = lane + 32 * i;

@@ -89,9 +89,9 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
   // workspace's per-unit chunk counters) and applies the append
   const bool fuse = sp.fuse_reduce != 0;
   const int L = max(p.seq_lens[b], 0);
-  int t0 = 0, t1 = L;
+  int t0 = p.first_token, t1 = L;
   if (split) {
-    t0 = c * p.chunk_tokens;
+    t0 = p.first_token + c * p.chunk_tokens;
     if (t0 >= L) {
       if (fuse && c == 0)  // empty sequence: its output rows are zero
         for (int i = tid; i < G * D; i += kWarps * 32) p.out[row0 * D + i] = __float2bfloat16_rn(0.f);
@@ -99,16 +99,20 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     }
     t1 = min(t0 + p.chunk_tokens, L);
   }
-  const int nch = split ? min((L + p.chunk_tokens - 1) / p.chunk_tokens, p.max_chunks) : 1;
+  const int nch = split ? min((L - p.first_token + p.chunk_tokens - 1) / p.chunk_tokens,
+                              p.max_chunks - p.chunk_slot0) : 1;
+  // first attended token of this unit: the chunk start, raised by the sliding window
+  const int lo = (p.window > 0 && L - p.window > t0) ? L - p.window : t0;
   int err = 0;
   if (static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
-      (split && static_cast<int64_t>(L) > static_cast<int64_t>(p.max_chunks) * p.chunk_tokens))
+      (split && static_cast<int64_t>(L - p.first_token) >
+                    static_cast<int64_t>(p.max_chunks - p.chunk_slot0) * p.chunk_tokens))
     err = PDA_DEV_BAD_SEQ_LEN;
 
   if (tid == 0) { cta_err[0] = 0; cta_err[1] = 0; }
-  const int n_tiles = err ? 0 : (t1 - t0 + kPageSize - 1) / kPageSize;
+  const int page0 = lo / kPageSize;  // first page touched (lo need not be page-aligned)
+  const int n_tiles = (err || lo >= t1) ? 0 : (t1 + kPageSize - 1) / kPageSize - page0;
   const int n_mine = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;  // tiles warp, warp+kWarps, ...
-  const int page0 = t0 / kPageSize;
 
   const uint32_t ring = smem_u32(smem + warp * C::kWarpRing);
   const uint32_t bar0 = smem_u32(bars + warp * kStages);
@@ -157,7 +161,24 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       if (lane == 0) issue(kk, page);
     }
   }
-  const bool append_here = sp.k_new != nullptr && !err && c == nch - 1;  // L > 0 here
+  const bool append_here = sp.k_new != nullptr && !err && L > 0 && c == nch - 1;
+  if (!kFp8 && append_here && n_tiles == 0 && warp == 0) {
+    // nothing of this unit is attended (the range starts past the new token): append only
+    const int v = table[(L - 1) / kPageSize];
+    if (v >= 0 && v < p.geom.num_pages) {
+      if (lane < C::kRowBytes / 16) {
+        const int64_t src = (static_cast<int64_t>(b) * p.geom.num_kv_heads + g) * D + lane * 8;
+        const int64_t dst = v * p.geom.page_stride + g * p.geom.head_stride +
+                            ((L - 1) % kPageSize) * p.geom.slot_stride + lane * 8;
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(sp.k_cache_w) + dst) =
+            *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(sp.k_new) + src);
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(sp.v_cache_w) + dst) =
+            *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(sp.v_new) + src);
+      }
+    } else {
+      bad_page = true;
+    }
+  }
 
   // ---- Q^T fragments (B operand of S^T = K.Q^T): column n = gid is head gid of the group
   uint32_t qf[C::kKSteps][2];
@@ -202,8 +223,9 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     const uint32_t bar = bar0 + 8 * s;
     if (!mbar_wait_bounded(bar, (kk / kStages) & 1)) { timed_out = true; break; }
     const uint32_t kt = ring + s * C::kStageBytes, vt = kt + C::kTileBytes;
-    const int tok0 = t0 + (warp + kk * kWarps) * kPageSize;
-    const int n_valid = min(kPageSize, t1 - tok0);
+    const int tok0 = (page0 + warp + kk * kWarps) * kPageSize;
+    const int n_valid = min(kPageSize, t1 - tok0);  // rows [n_skip, n_valid) of the tile are attended
+    const int n_skip = max(lo - tok0, 0);           // > 0 only in the unit's first tile
     float ksc = 1.f, vsc = 1.f;
     if (kFp8) {
       ksc = __shfl_sync(0xffffffffu, ksA, kk & 31);
@@ -229,11 +251,14 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       __syncwarp();
     }
-    if (n_valid < kPageSize) {
-      // rows past the sequence end may hold anything: clear them in V (K is masked by select)
+    if (n_valid < kPageSize || n_skip > 0) {
+      // rows outside the attended range may hold anything: clear them in V (K is masked by select)
       const int n_chunks = C::kRowBytes / 16;
-      for (int i = lane; i < (kPageSize - n_valid) * n_chunks; i += 32) {
-        const int r = n_valid + i / n_chunks, ch = i % n_chunks;
+      const int n_clear = kPageSize - n_valid + n_skip;
+      for (int i = lane; i < n_clear * n_chunks; i += 32) {
+        int r = i / n_chunks;
+        const int ch = i % n_chunks;
+        r = r < n_skip ? r : n_valid + (r - n_skip);
         asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_off(r, ch)), "r"(0));
       }
       __syncwarp();
@@ -265,9 +290,9 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     const float sc = scale_log2 * ksc;
     float s0 = (sa[0] + sb[0]) * sc, s1 = (sa[1] + sb[1]) * sc;   // token gid,   heads 2tq, 2tq+1
     float s2 = (sa[2] + sb[2]) * sc, s3 = (sa[3] + sb[3]) * sc;   // token gid+8
-    if (n_valid < kPageSize) {
-      if (gid >= n_valid) { s0 = -INFINITY; s1 = -INFINITY; }
-      if (gid + 8 >= n_valid) { s2 = -INFINITY; s3 = -INFINITY; }
+    if (n_valid < kPageSize || n_skip > 0) {
+      if (gid >= n_valid || gid < n_skip) { s0 = -INFINITY; s1 = -INFINITY; }
+      if (gid + 8 >= n_valid || gid + 8 < n_skip) { s2 = -INFINITY; s3 = -INFINITY; }
     }
 
     // ---- online softmax (base 2), max over the tile's tokens = over gid and the two rows
@@ -277,7 +302,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
     }
-    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: token 0 of a tile is always valid
+    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: every tile has an attended row
     const float al0 = ex2(m0 - mn0), al1 = ex2(m1 - mn1);     // ex2(-inf) = 0 on the first tile
     m0 = mn0; m1 = mn1;
     const float p0 = ex2(s0 - mn0), p1 = ex2(s1 - mn1), p2 = ex2(s2 - mn0), p3 = ex2(s3 - mn1);
@@ -398,7 +423,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     const bool live = !dev_err && lsum > 0.f;
     const float val = live ? acc / lsum : 0.f;
     if (split && !(fuse && nch == 1)) {
-      const int64_t pr = (row0 + h) * p.max_chunks + c;
+      const int64_t pr = (row0 + h) * p.max_chunks + p.chunk_slot0 + c;
       p.part_o[pr * D + d] = val;
       if (d == 0) p.part_lse[pr] = live ? (M + __log2f(lsum)) * kLn2 : -INFINITY;
     } else {
@@ -419,12 +444,12 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       for (int idx = tid; idx < G * D; idx += kWarps * 32) {
         const int h = idx / D, d = idx % D;
         const int64_t row = row0 + h;
-        const float* lse = p.part_lse + row * p.max_chunks;
+        const float* lse = p.part_lse + row * p.max_chunks + p.chunk_slot0;
         float M = -INFINITY;
         for (int cc = 0; cc < nch; ++cc) M = fmaxf(M, __ldcg(lse + cc));
         float acc = 0.f, W = 0.f;
         if (M > -INFINITY) {
-          const float* po = p.part_o + row * p.max_chunks * D + d;
+          const float* po = p.part_o + (row * p.max_chunks + p.chunk_slot0) * D + d;
           for (int cc = 0; cc < nch; ++cc) {
             const float w = __expf(__ldcg(lse + cc) - M);
             W += w;

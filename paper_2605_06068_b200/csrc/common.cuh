@@ -33,6 +33,10 @@ struct AttnParams {
   int32_t block_table_stride, batch, num_q_heads, group;  // group = Hq / Hkv
   int32_t chunk_tokens, max_chunks;
   float scale;
+  // Token range: tokens below max(first_token, L - window) are not attended (window <= 0: no
+  // window). Chunk c covers [first_token + c*chunk_tokens, ...) and is stored in partial slot
+  // chunk_slot0 + c. first_token is a multiple of the page size.
+  int32_t window, first_token, chunk_slot0;
 };
 
 // Fused decode step (attention_tma.cu): attention parameters plus the
@@ -86,8 +90,8 @@ bool attention_tma_supports(const AttnParams& p);
 cudaError_t launch_step_tma(const StepParams& sp, cudaStream_t stream);
 cudaError_t launch_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
                           int32_t batch, int32_t num_q_heads, int32_t head_dim,
-                          int32_t chunk_tokens, int32_t max_chunks, __nv_bfloat16* out,
-                          cudaStream_t stream);
+                          int32_t chunk_tokens, int32_t max_chunks, int32_t first_token,
+                          int32_t first_chunks, __nv_bfloat16* out, cudaStream_t stream);
 cudaError_t launch_e4m3_decode(float* out256, cudaStream_t stream);
 
 }  // namespace pda

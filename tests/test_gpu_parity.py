@@ -429,3 +429,40 @@ def test_step_host_matches_device_calls(oracle):
         assert_close(got, ref, what=f"step_host chunk {chunk}")
         k_ref, _ = host_appended(oracle, w)
         assert (bf16_to_bits(dw.k_cache) == k_ref).all()
+
+
+# ---- sliding window -------------------------------------------------------------------------
+
+@pytest.mark.parametrize("flags", PATHS)
+@pytest.mark.parametrize("shape", [(8, 2, 64), (32, 8, 128)])
+def test_sliding_window(oracle, flags, shape):
+    Hq, Hkv, D = shape
+    lens = [1, 15, 16, 17, 40, 100, 333, 1000]
+    w = W.make_workload("win", lens, Hq, Hkv, D, seed=61)
+    dw = DeviceWorkload(w)
+    dw.append()
+    k, v = host_appended(oracle, w)
+    for window in (1, 7, 16, 33, 128, 5000):
+        ref, _ = oracle.paged_decode_attention(w.q, k, v, w.block_table, w.seq_lens, w.scale, window=window)
+        # pages wholly before the window may be evicted: poison their table entries
+        bt = dw.block_table.clone()
+        for b, L in enumerate(lens):
+            first_live = max(0, L - window) // 16
+            bt[b, :first_live] = -7
+        out = pda.paged_window_decode_attention(dw.q, dw.k_cache, dw.v_cache, bt, dw.seq_lens,
+                                                float(w.scale), window, flags=flags, status=dw.status)
+        assert_close(bf16_to_f64(out), ref, what=f"window {window} unsplit")
+        if window == 1:   # the last V row, bit for bit
+            got = bf16_to_bits(out)
+            for b in range(len(lens)):
+                assert (got[b, 0] == w.v_new[b, 0]).all()
+        for chunk in (32, 256):
+            mc = pda.max_chunks(max(lens), chunk)
+            po = torch.full((w.batch, Hq, mc, D), float("nan"), dtype=torch.float32, device="cuda")
+            pl = torch.full((w.batch, Hq, mc), float("nan"), dtype=torch.float32, device="cuda")
+            pda.paged_window_decode_attention(dw.q, dw.k_cache, dw.v_cache, bt, dw.seq_lens, float(w.scale),
+                                              window, chunk_tokens=chunk, part_o=po, part_lse=pl, flags=flags,
+                                              status=dw.status)
+            out_s = pda.paged_decode_reduce(po, pl, dw.seq_lens, chunk)
+            assert_close(bf16_to_f64(out_s), ref, what=f"window {window} chunk {chunk}")
+    assert status_of(dw) == 0

@@ -347,3 +347,34 @@ def test_fp8_attention_matches_library_sdpa_on_dequantised_cache(oracle):
     np.testing.assert_allclose(out, ref, rtol=0, atol=1e-12)
     # all rows alias the same prefix pages
     assert (w.block_table[:, :128] == w.block_table[0, :128]).all()
+
+
+# ---- sliding window ----------------------------------------------------------------------
+
+@pytest.mark.parametrize("window", [1, 5, 16, 17, 40, 1000])
+def test_window_matches_library_sdpa_on_the_last_tokens(oracle, window):
+    w = W.tiny(seed=42)
+    k, v = appended(oracle, w)
+    out, lse = oracle.paged_decode_attention(w.q, k, v, w.block_table, w.seq_lens, w.scale, window=window)
+    G = w.num_q_heads // w.num_kv_heads
+    for b in range(w.batch):
+        K, V = dense_kv(w, k, v, b)
+        lo = max(0, int(w.seq_lens[b]) - window)
+        q = torch.from_numpy(W.bf16_bits_to_f32(w.q[b]).astype(np.float64))[None, :, None, :]
+        Kt = torch.from_numpy(K[:, lo:]).repeat_interleave(G, dim=0)[None]
+        Vt = torch.from_numpy(V[:, lo:]).repeat_interleave(G, dim=0)[None]
+        o = torch.nn.functional.scaled_dot_product_attention(q, Kt, Vt, scale=float(w.scale))
+        np.testing.assert_allclose(out[b], o[0, :, 0, :].numpy(), rtol=0, atol=1e-12)
+    # window = 1 returns the last V row exactly; a window covering everything changes nothing
+    if window == 1:
+        for b in range(w.batch):
+            assert (out[b, 0] == W.bf16_bits_to_f32(w.v_new[b, 0]).astype(np.float64)).all()
+    if window == 1000:
+        full, _ = oracle.paged_decode_attention(w.q, k, v, w.block_table, w.seq_lens, w.scale)
+        assert (out == full).all()
+    # split + reduce under a window equals the unsplit windowed result
+    po, pl = oracle.paged_decode_attention(w.q, k, v, w.block_table, w.seq_lens, w.scale,
+                                           chunk_tokens=32, max_chunks=4, window=window)
+    out2, lse2 = oracle.paged_decode_reduce(po, pl, w.seq_lens, 32)
+    np.testing.assert_allclose(out2, out, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse2, lse, rtol=0, atol=1e-12)
