@@ -161,6 +161,64 @@ int paged_window_decode_attention(const void* q, const void* k_cache, const void
                                   int32_t max_chunks, uint32_t flags, int32_t* status,
                                   pda_stream_t stream);
 
+/* Append of n_new tokens per sequence (the draft block of a verification step):
+ * k_new, v_new are [batch, n_new, num_kv_heads, head_dim] bf16; token i becomes
+ * logical token seq_lens[b] - n_new + i (seq_lens = length AFTER the append).
+ * n_new == 1 is kv_append. */
+int kv_append_tokens(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                     const pda_cache_desc* desc, const int32_t* block_table,
+                     int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+                     int32_t n_new, int32_t* status, pda_stream_t stream);
+
+/* Verification attention over a block of n_query_tokens draft tokens per sequence
+ * (the predicted-output verifier of the paper scores 16-token blocks in one pass:
+ * Section 4.2 and Appendix A, Scenario B; the paper prints no formula -- this is
+ * causal attention over the paged cache). The cache already holds all seq_lens[b]
+ * tokens, the block being the last n_query_tokens of them; query token i stands at
+ * position L - n + i and attends tokens j <= L - n + i.
+ *   q, out    [batch, n_query_tokens, num_q_heads, head_dim] bf16
+ *   chunk_tokens 0: one unit per (sequence, kv head).  > 0: split-KV; the partials
+ *             part_o [batch, n, num_q_heads, max_chunks, head_dim] and part_lse
+ *             [batch, n, num_q_heads, max_chunks] are scratch and the merge runs
+ *             inside this call.  `out` is always written.
+ * The query rows of a kv head's group form dense tensor-core tiles (rows = tokens x
+ * group size), so each page is fetched once per block, not once per token.
+ * Supported: head_dim 64 or 128 (bf16), 128 (e4m3). */
+int paged_verify_attention(const void* q, const void* k_cache, const void* v_cache,
+                           const pda_cache_desc* desc, const float* k_scale,
+                           const float* v_scale, const int32_t* block_table,
+                           int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+                           int32_t num_q_heads, int32_t n_query_tokens, float scale,
+                           int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                           int32_t max_chunks, int32_t* status, pda_stream_t stream);
+
+/* Decode attention for a batch whose sequences all start with the SAME
+ * prefix_tokens tokens stored in the same physical pages (the shared-prefix
+ * prompt-caching workload of the paper: Section 4.2 and Appendix A, Scenario C).
+ * The result is exactly paged_decode_attention's; the work is reorganised: the
+ * prefix's keys/values are read once for the whole batch (all queries of a kv
+ * head's groups as one block of rows), each sequence's own suffix is attended
+ * separately, and the pieces are merged by their log-sum-exp weights.
+ *   block_table    rows must agree on their first prefix_tokens/page_size entries
+ *                  (row 0's are used); prefix_tokens is a multiple of page_size and
+ *                  <= every seq_lens[b]
+ *   prefix_chunk_tokens  split of the prefix for parallelism (multiple of page_size)
+ *   chunk_tokens   (> 0) split of the suffixes
+ *   part_o, part_lse  scratch [batch, num_q_heads, max_chunks, head_dim] / [.., max_chunks]
+ *                  with max_chunks >= ceil(prefix_tokens/prefix_chunk_tokens)
+ *                                    + ceil((max seq_len - prefix_tokens)/chunk_tokens)
+ *   out            [batch, num_q_heads, head_dim] bf16
+ * Three launches on `stream` (prefix, suffixes, merge). Supported: group size <= 8,
+ * head_dim 64/128 (bf16) or 128 (e4m3), batch <= 4096. */
+int paged_prefix_decode_attention(const void* q, const void* k_cache, const void* v_cache,
+                                  const pda_cache_desc* desc, const float* k_scale,
+                                  const float* v_scale, const int32_t* block_table,
+                                  int32_t block_table_stride, const int32_t* seq_lens,
+                                  int32_t batch, int32_t num_q_heads, float scale,
+                                  int32_t prefix_tokens, int32_t prefix_chunk_tokens,
+                                  int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                                  int32_t max_chunks, int32_t* status, pda_stream_t stream);
+
 /* Merge of split-KV partials (the reduce step of flash-decoding; exact algebra):
  *     out[b,h,:] = sum_c w_c part_o[b,h,c,:] / sum_c w_c,
  *     w_c = exp(part_lse[b,h,c] - max_c part_lse[b,h,c]),  c < ceil(L_b/chunk_tokens)

@@ -128,6 +128,49 @@ def paged_decode_attention(q, k_cache, v_cache, block_table, seq_lens, scale,
     return out, lse
 
 
+def kv_append_tokens(k_new, v_new, k_cache, v_cache, block_table, seq_lens):
+    """In-place append of ``n_new`` tokens per sequence; ``k_new`` is ``[B,n_new,Hkv,D]``."""
+    assert k_cache.dtype == np.uint16 and k_new.dtype == np.uint16 and k_new.ndim == 4
+    k_new, v_new = np.ascontiguousarray(k_new), np.ascontiguousarray(v_new)
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    ps, hs, ss = _cache_strides(k_cache)
+    _, Hkv, P, D = k_cache.shape
+    _load().oracle_kv_append_tokens(
+        _p(k_new), _p(v_new), _p(k_cache), _p(v_cache), C.c_int64(ps), C.c_int64(hs),
+        C.c_int64(ss), C.c_int32(P), C.c_int32(Hkv), C.c_int32(D), C.c_int32(2),
+        _p(block_table), C.c_int32(block_table.shape[1]), _p(seq_lens),
+        C.c_int32(seq_lens.shape[0]), C.c_int32(k_new.shape[1]))
+
+
+def paged_verify_attention(q, k_cache, v_cache, block_table, seq_lens, scale,
+                           k_scale=None, v_scale=None, n_threads=0):
+    """Causal attention of a block of query tokens: ``q [B,T,Hq,D]`` -> ``(out, lse)`` fp64;
+    query ``i`` attends tokens ``j <= L - T + i`` (the cache already holds the block)."""
+    q = np.ascontiguousarray(q)
+    assert q.dtype == np.uint16 and q.ndim == 4
+    B, T, Hq, D = q.shape
+    dtype = 0 if k_cache.dtype == np.uint16 else 1
+    if dtype == 1:
+        k_scale = np.ascontiguousarray(k_scale, dtype=np.float32)
+        v_scale = np.ascontiguousarray(v_scale, dtype=np.float32)
+    ps, hs, ss = _cache_strides(k_cache)
+    _, Hkv, P, _ = k_cache.shape
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    out = np.zeros((B, T, Hq, D), dtype=np.float64)
+    lse = np.zeros((B, T, Hq), dtype=np.float64)
+    if n_threads <= 0:
+        n_threads = hardware_threads()
+    _load().oracle_paged_verify_attention(
+        _p(q), _p(k_cache), _p(v_cache), C.c_int32(dtype), _p(k_scale), _p(v_scale),
+        C.c_int64(ps), C.c_int64(hs), C.c_int64(ss), C.c_int32(P), C.c_int32(Hkv), C.c_int32(D),
+        _p(block_table), C.c_int32(block_table.shape[1]), _p(seq_lens), C.c_int32(B),
+        C.c_int32(Hq), C.c_int32(T), C.c_float(np.float32(scale)), _p(out), _p(lse),
+        C.c_int32(n_threads))
+    return out, lse
+
+
 def paged_decode_reduce(part_o, part_lse, seq_lens, chunk_tokens):
     """Merge ``[B,Hq,C,D]`` / ``[B,Hq,C]`` partials; returns ``(out, lse)`` fp64."""
     part_o = np.ascontiguousarray(part_o, dtype=np.float64)

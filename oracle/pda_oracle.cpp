@@ -227,6 +227,62 @@ void oracle_paged_decode_attention(
   });
 }
 
+// Append of n_new tokens per sequence: token i of new[b] (rows [B, n_new, Hkv, D])
+// becomes logical token L_b - n_new + i, bytewise.
+void oracle_kv_append_tokens(const uint8_t* k_new, const uint8_t* v_new, uint8_t* k_cache,
+                             uint8_t* v_cache, int64_t page_stride, int64_t head_stride,
+                             int64_t slot_stride, int32_t page_size, int32_t num_kv_heads,
+                             int32_t head_dim, int32_t elem_bytes, const int32_t* block_table,
+                             int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+                             int32_t n_new) {
+  for (int b = 0; b < batch; ++b) {
+    const int64_t L = seq_lens[b];
+    for (int i = 0; i < n_new; ++i) {
+      const int64_t pos = L - n_new + i;
+      if (L <= 0 || pos < 0) continue;
+      const int64_t page = block_table[static_cast<int64_t>(b) * block_table_stride + pos / page_size];
+      const int64_t slot = pos % page_size;
+      for (int g = 0; g < num_kv_heads; ++g) {
+        const int64_t dst = (page * page_stride + g * head_stride + slot * slot_stride) * elem_bytes;
+        const int64_t src = ((static_cast<int64_t>(b) * n_new + i) * num_kv_heads + g) * head_dim * elem_bytes;
+        std::memcpy(k_cache + dst, k_new + src, static_cast<size_t>(head_dim) * elem_bytes);
+        std::memcpy(v_cache + dst, v_new + src, static_cast<size_t>(head_dim) * elem_bytes);
+      }
+    }
+  }
+}
+
+// Verification attention for a block of n_q query tokens per sequence (the
+// predicted-output verifier of the paper's Scenario B scores a 16-token block
+// in one pass; the paper gives no formula -- this is causal attention written
+// out): the cache already holds all L_b tokens, the block being its last n_q;
+// query token i stands at position L_b - n_q + i and attends tokens
+// j <= L_b - n_q + i. q and out are [B, n_q, Hq, D], lse is [B, n_q, Hq].
+void oracle_paged_verify_attention(
+    const uint16_t* q, const uint8_t* k_cache, const uint8_t* v_cache, int32_t kv_dtype,
+    const float* k_scale, const float* v_scale, int64_t page_stride, int64_t head_stride,
+    int64_t slot_stride, int32_t page_size, int32_t num_kv_heads, int32_t head_dim,
+    const int32_t* block_table, int32_t block_table_stride, const int32_t* seq_lens,
+    int32_t batch, int32_t num_q_heads, int32_t n_q, float scale, double* out, double* lse,
+    int32_t n_threads) {
+  const int G = num_q_heads / num_kv_heads;
+  const CacheView K{k_cache, kv_dtype, page_stride, head_stride, slot_stride, k_scale, num_kv_heads};
+  const CacheView V{v_cache, kv_dtype, page_stride, head_stride, slot_stride, v_scale, num_kv_heads};
+  const double sc = static_cast<double>(scale);
+  const int64_t rows = static_cast<int64_t>(batch) * n_q * num_q_heads;
+  parallel_for(rows, n_threads, [&](int64_t row) {
+    const int h = static_cast<int>(row % num_q_heads);
+    const int i = static_cast<int>((row / num_q_heads) % n_q);
+    const int b = static_cast<int>(row / (static_cast<int64_t>(num_q_heads) * n_q));
+    const int64_t L = seq_lens[b] > 0 ? seq_lens[b] : 0;
+    int64_t limit = L - n_q + i + 1;  // number of visible tokens
+    if (limit < 0) limit = 0;
+    if (limit > L) limit = L;
+    attend_range(q + row * head_dim, K, V, block_table + static_cast<int64_t>(b) * block_table_stride,
+                 page_size, head_dim, h / G, sc, 0, limit, out + row * head_dim, lse + row);
+  });
+}
+
 // Merge of split-KV partials: each chunk's o_c is already normalised within the
 // chunk and lse_c = m_c + log(l_c), so the full softmax average is
 //   out = sum_c w_c o_c / sum_c w_c,  w_c = exp(lse_c - max_c lse_c).

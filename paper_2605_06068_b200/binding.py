@@ -22,7 +22,8 @@ DEV_STATUS = {0: "ok", 1: "bad page id", 2: "seq_len exceeds block table", 3: "c
 EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
            "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
-           "paged_decode_step", "pda_advance_seq_lens", "paged_window_decode_attention"]
+           "paged_decode_step", "pda_advance_seq_lens", "paged_window_decode_attention", "kv_append_tokens",
+           "paged_verify_attention", "paged_prefix_decode_attention"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
@@ -56,6 +57,11 @@ def lib():
         L.paged_decode_step_host.argtypes = [vp] * 5 + [vp] * 5 + [vp, vp, dp, i32, i32, i32, f32,
                                                                  i32, vp, vp, i32, vp, vp, vp, vp, vp]
         L.pda_workspace_ints.argtypes = [i32, i32]
+        L.kv_append_tokens.argtypes = [vp, vp, vp, vp, dp, vp, i32, vp, i32, i32, vp, vp]
+        L.paged_verify_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, i32, f32,
+                                             i32, vp, vp, vp, i32, vp, vp]
+        L.paged_prefix_decode_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
+                                                    i32, i32, i32, vp, vp, vp, i32, vp, vp]
         L.paged_window_decode_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
                                                     i32, i32, vp, vp, vp, i32, u32, vp, vp]
         L.pda_advance_seq_lens.argtypes = [vp, i32, i32, vp]
@@ -252,3 +258,53 @@ def advance_seq_lens(seq_lens, delta=1, stream=None):
     """``seq_lens += delta`` on the device, in stream order (graph-capturable)."""
     _check(lib().pda_advance_seq_lens(_ptr(seq_lens), seq_lens.shape[0], int(delta), _stream(stream)),
            "pda_advance_seq_lens")
+
+
+def kv_append_tokens(k_new, v_new, k_cache, v_cache, block_table, seq_lens, status=None, stream=None):
+    """Append ``k_new``/``v_new`` ``[B,n_new,Hkv,D]``; ``seq_lens`` is the length after the append."""
+    desc = cache_desc(k_cache)
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.dim() == 4
+    rc = lib().kv_append_tokens(_ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), C.byref(desc),
+                                _ptr(block_table), block_table.stride(0), _ptr(seq_lens),
+                                seq_lens.shape[0], k_new.shape[1], _ptr(status), _stream(stream))
+    _check(rc, "kv_append_tokens")
+
+
+def paged_verify_attention(q, k_cache, v_cache, block_table, seq_lens, scale, chunk_tokens=0, out=None,
+                           part_o=None, part_lse=None, k_scale=None, v_scale=None, status=None,
+                           stream=None):
+    """Causal attention of a block of query tokens ``q [B,T,Hq,D]``; returns ``out [B,T,Hq,D]``."""
+    desc = cache_desc(k_cache)
+    assert q.is_contiguous() and q.dim() == 4
+    B, T, Hq, D = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    mc = 0
+    if chunk_tokens:
+        mc = part_o.shape[3]
+        assert tuple(part_o.shape) == (B, T, Hq, mc, D) and tuple(part_lse.shape) == (B, T, Hq, mc)
+    rc = lib().paged_verify_attention(
+        _ptr(q), _ptr(k_cache), _ptr(v_cache), C.byref(desc), _ptr(k_scale), _ptr(v_scale),
+        _ptr(block_table), block_table.stride(0), _ptr(seq_lens), B, Hq, T, float(scale),
+        chunk_tokens, _ptr(out), _ptr(part_o), _ptr(part_lse), mc, _ptr(status), _stream(stream))
+    _check(rc, "paged_verify_attention")
+    return out
+
+
+def paged_prefix_decode_attention(q, k_cache, v_cache, block_table, seq_lens, scale, prefix_tokens,
+                                  prefix_chunk_tokens, chunk_tokens, part_o, part_lse, out=None,
+                                  k_scale=None, v_scale=None, status=None, stream=None):
+    """Decode attention of a batch sharing its first ``prefix_tokens`` tokens' pages."""
+    desc = cache_desc(k_cache)
+    B, Hq, D = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    mc = part_o.shape[2]
+    assert tuple(part_o.shape) == (B, Hq, mc, D) and tuple(part_lse.shape) == (B, Hq, mc)
+    rc = lib().paged_prefix_decode_attention(
+        _ptr(q), _ptr(k_cache), _ptr(v_cache), C.byref(desc), _ptr(k_scale), _ptr(v_scale),
+        _ptr(block_table), block_table.stride(0), _ptr(seq_lens), B, Hq, float(scale),
+        int(prefix_tokens), int(prefix_chunk_tokens), int(chunk_tokens), _ptr(out), _ptr(part_o),
+        _ptr(part_lse), mc, _ptr(status), _stream(stream))
+    _check(rc, "paged_prefix_decode_attention")
+    return out

@@ -174,6 +174,102 @@ int paged_window_decode_attention(const void* q, const void* k_cache, const void
   return static_cast<int>(pda::launch_attention_generic(p, s));
 }
 
+int kv_append_tokens(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                     const pda_cache_desc* desc, const int32_t* block_table,
+                     int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+                     int32_t n_new, int32_t* status, pda_stream_t stream) {
+  CacheGeom g;
+  if (int rc = check_desc(desc, &g)) return rc;
+  if (g.dtype != PDA_BF16) return PDA_ERR_UNSUPPORTED;
+  if (batch < 0 || block_table_stride < 0 || n_new < 0) return PDA_ERR_INVALID_ARG;
+  if (batch == 0 || n_new == 0) return PDA_OK;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !seq_lens ||
+      block_table_stride == 0)
+    return PDA_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache))
+    return PDA_ERR_MISALIGNED;
+  return static_cast<int>(pda::launch_kv_append_tokens(k_new, v_new, k_cache, v_cache, g,
+                                                       block_table, block_table_stride, seq_lens,
+                                                       batch, n_new, status,
+                                                       static_cast<cudaStream_t>(stream)));
+}
+
+int paged_verify_attention(const void* q, const void* k_cache, const void* v_cache,
+                           const pda_cache_desc* desc, const float* k_scale,
+                           const float* v_scale, const int32_t* block_table,
+                           int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
+                           int32_t num_q_heads, int32_t n_query_tokens, float scale,
+                           int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                           int32_t max_chunks, int32_t* status, pda_stream_t stream) {
+  AttnParams p;
+  if (n_query_tokens <= 0 || n_query_tokens > 4096) return PDA_ERR_INVALID_ARG;
+  if (!out && batch > 0) return PDA_ERR_INVALID_ARG;
+  if (int rc = check_attention(q, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                               block_table_stride, seq_lens, batch, num_q_heads, chunk_tokens,
+                               out, part_o, part_lse, max_chunks, &p))
+    return rc;
+  if (static_cast<int64_t>(batch) * n_query_tokens > 65535) return PDA_ERR_TOO_LARGE;
+  if (batch == 0) return PDA_OK;
+  p.status = status;
+  p.scale = scale;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  pda::MqParams mp{p, n_query_tokens, 1, 0, max_chunks};
+  if (!pda::attention_mq_supports(mp)) return PDA_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaError_t e = pda::launch_attention_mq(mp, s)) return static_cast<int>(e);
+  if (chunk_tokens > 0)
+    return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
+                                               p.geom.head_dim, chunk_tokens, max_chunks, 0, 0,
+                                               n_query_tokens, static_cast<__nv_bfloat16*>(out), s));
+  return PDA_OK;
+}
+
+int paged_prefix_decode_attention(const void* q, const void* k_cache, const void* v_cache,
+                                  const pda_cache_desc* desc, const float* k_scale,
+                                  const float* v_scale, const int32_t* block_table,
+                                  int32_t block_table_stride, const int32_t* seq_lens,
+                                  int32_t batch, int32_t num_q_heads, float scale,
+                                  int32_t prefix_tokens, int32_t prefix_chunk_tokens,
+                                  int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
+                                  int32_t max_chunks, int32_t* status, pda_stream_t stream) {
+  AttnParams p;
+  if (prefix_tokens <= 0 || prefix_chunk_tokens <= 0 || chunk_tokens <= 0) return PDA_ERR_INVALID_ARG;
+  if (prefix_tokens % pda::kPageSize || prefix_chunk_tokens % pda::kPageSize) return PDA_ERR_INVALID_ARG;
+  if (!out && batch > 0) return PDA_ERR_INVALID_ARG;
+  if (int rc = check_attention(q, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                               block_table_stride, seq_lens, batch, num_q_heads, chunk_tokens,
+                               out, part_o, part_lse, max_chunks, &p))
+    return rc;
+  const int prefix_chunks = (prefix_tokens + prefix_chunk_tokens - 1) / prefix_chunk_tokens;
+  if (prefix_chunks >= max_chunks) return PDA_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(prefix_tokens) > static_cast<int64_t>(block_table_stride) * pda::kPageSize)
+    return PDA_ERR_INVALID_ARG;
+  if (batch == 0) return PDA_OK;
+  p.status = status;
+  p.scale = scale;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  // (1) the shared prefix once: the batch's queries as one block of rows per kv head
+  AttnParams pp = p;
+  pp.batch = 1;
+  pp.chunk_tokens = prefix_chunk_tokens;
+  pp.chunk_slot0 = 0;
+  pda::MqParams mp{pp, batch, 0, prefix_tokens, prefix_chunks};
+  if (!pda::attention_mq_supports(mp) || !pda::attention_tma_supports(p)) return PDA_ERR_UNSUPPORTED;
+  if (cudaError_t e = pda::launch_attention_mq(mp, s)) return static_cast<int>(e);
+  // (2) every sequence's own suffix, chunk slots after the prefix's
+  AttnParams ps = p;
+  ps.first_token = prefix_tokens;
+  ps.chunk_slot0 = prefix_chunks;
+  if (cudaError_t e = pda::launch_attention_tma(ps, s)) return static_cast<int>(e);
+  // (3) merge
+  return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
+                                             p.geom.head_dim, chunk_tokens, max_chunks,
+                                             prefix_tokens, prefix_chunks, 1,
+                                             static_cast<__nv_bfloat16*>(out), s));
+}
+
 int pda_workspace_ints(int32_t batch, int32_t num_kv_heads) {
   if (batch < 0 || num_kv_heads <= 0) return PDA_ERR_INVALID_ARG;
   const int64_t n = 2 + static_cast<int64_t>(batch) * num_kv_heads;
@@ -232,7 +328,7 @@ int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_
   if (batch == 0) return PDA_OK;
   if (!part_o || !part_lse || !seq_lens || !out) return PDA_ERR_INVALID_ARG;
   return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
-                                             head_dim, chunk_tokens, max_chunks, 0, 0,
+                                             head_dim, chunk_tokens, max_chunks, 0, 0, 1,
                                              static_cast<__nv_bfloat16*>(out),
                                              static_cast<cudaStream_t>(stream)));
 }

@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(32) attention_generic_kernel(AttnParams p) {
 
 cudaError_t launch_attention_generic(const AttnParams& p, cudaStream_t stream) {
   if (p.batch == 0 || p.num_q_heads == 0) return cudaSuccess;
-  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks) : 1u;
+  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks - p.chunk_slot0) : 1u;
   dim3 grid(chunks, p.num_q_heads, p.batch);
   if (p.geom.dtype == PDA_FP8_E4M3)
     attention_generic_kernel<true><<<grid, 32, 0, stream>>>(p);

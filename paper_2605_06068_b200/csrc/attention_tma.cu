@@ -480,7 +480,7 @@ cudaError_t launch(const StepParams& sp, cudaStream_t stream) {
   auto kern = attention_tma_kernel<D, kFp8, kStages, kWarps>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
-  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks) : 1u;
+  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks - p.chunk_slot0) : 1u;
   dim3 grid(chunks, p.geom.num_kv_heads, p.batch);
   kern<<<grid, kWarps * 32, C::kSmemBytes, stream>>>(k_map, v_map, sp);
   return cudaGetLastError();

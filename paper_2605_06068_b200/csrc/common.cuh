@@ -51,6 +51,15 @@ struct StepParams {
   int32_t fuse_reduce; // 1: the launch writes `out` itself (needs workspace when split)
 };
 
+// Multi-query attention (attention_mq.cu): n_q query tokens per sequence.
+struct MqParams {
+  AttnParams a;           // q is [B, n_q, Hq, D]; out / partials are indexed by (b*n_q + i)
+  int32_t n_q;            // query tokens per sequence
+  int32_t causal;         // 1: query i sees keys j < L - n_q + i + 1
+  int32_t kv_len_fixed;   // > 0: every sequence attends [first_token, kv_len_fixed) (shared prefix)
+  int32_t n_chunks_grid;  // chunk CTAs launched per (sequence, head) when split
+};
+
 __device__ __forceinline__ void report(int32_t* status, int code) {
   if (status != nullptr) atomicMax(status, code);
 }
@@ -88,10 +97,18 @@ cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream);
 bool attention_tma_supports(const AttnParams& p);
 // Fused step on the same kernel: optional append, optional in-kernel reduce (sp.fuse_reduce).
 cudaError_t launch_step_tma(const StepParams& sp, cudaStream_t stream);
+// Rows are (sequence, query token, head): tokens_per_seq query tokens share one seq_lens entry.
 cudaError_t launch_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
                           int32_t batch, int32_t num_q_heads, int32_t head_dim,
                           int32_t chunk_tokens, int32_t max_chunks, int32_t first_token,
-                          int32_t first_chunks, __nv_bfloat16* out, cudaStream_t stream);
+                          int32_t first_chunks, int32_t tokens_per_seq, __nv_bfloat16* out,
+                          cudaStream_t stream);
+bool attention_mq_supports(const MqParams& mp);
+cudaError_t launch_attention_mq(const MqParams& mp, cudaStream_t stream);
+cudaError_t launch_kv_append_tokens(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                    const CacheGeom& g, const int32_t* block_table, int32_t bt_stride,
+                                    const int32_t* seq_lens, int32_t batch, int32_t n_new,
+                                    int32_t* status, cudaStream_t stream);
 cudaError_t launch_e4m3_decode(float* out256, cudaStream_t stream);
 
 }  // namespace pda

@@ -1,0 +1,113 @@
+"""GPU parity of the multi-query kernel's two uses: verification attention over a
+block of draft tokens (causal inside the block) and the shared-prefix cascade."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_06068_b200 import binding as pda
+from paper_2605_06068_b200 import workloads as W
+
+from util import DeviceWorkload, assert_close, bf16_tensor, bf16_to_bits, bf16_to_f64, oracle_out
+
+pytestmark = pytest.mark.gpu
+
+
+def verify_inputs(w, T, seed):
+    rng = np.random.default_rng(seed)
+    B = w.batch
+    q = W.f32_to_bf16_bits(rng.standard_normal((B, T, w.num_q_heads, w.head_dim), dtype=np.float32))
+    kn = W.f32_to_bf16_bits(rng.standard_normal((B, T, w.num_kv_heads, w.head_dim), dtype=np.float32))
+    vn = W.f32_to_bf16_bits(rng.standard_normal((B, T, w.num_kv_heads, w.head_dim), dtype=np.float32))
+    return q, kn, vn
+
+
+@pytest.mark.parametrize("T", [1, 4, 16])
+@pytest.mark.parametrize("shape", [(8, 2, 64), (32, 8, 128), (64, 8, 128), (8, 8, 128)],
+                         ids=lambda s: f"Hq{s[0]}kv{s[1]}D{s[2]}")
+def test_verify_attention_and_block_append(oracle, shape, T):
+    Hq, Hkv, D = shape
+    lens = [16, 17, 31, 40, 100, 640, 1300]
+    w = W.make_workload("verify", lens, Hq, Hkv, D, seed=19)
+    q, kn, vn = verify_inputs(w, T, 20)
+    k, v = w.k_cache.copy(), w.v_cache.copy()
+    oracle.kv_append_tokens(kn, vn, k, v, w.block_table, w.seq_lens)
+    ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
+
+    dw = DeviceWorkload(w)
+    pda.kv_append_tokens(bf16_tensor(kn), bf16_tensor(vn), dw.k_cache, dw.v_cache, dw.block_table,
+                         dw.seq_lens, status=dw.status)
+    assert (bf16_to_bits(dw.k_cache) == k).all() and (bf16_to_bits(dw.v_cache) == v).all()
+    dq = bf16_tensor(q)
+    out = pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                     float(w.scale), status=dw.status)
+    assert_close(bf16_to_f64(out), ref, what=f"verify T={T} unsplit")
+    for chunk in (64, 256):
+        mc = pda.max_chunks(max(lens), chunk)
+        po = torch.full((w.batch, T, Hq, mc, D), float("nan"), dtype=torch.float32, device="cuda")
+        pl = torch.full((w.batch, T, Hq, mc), float("nan"), dtype=torch.float32, device="cuda")
+        out_s = pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                           float(w.scale), chunk_tokens=chunk, part_o=po, part_lse=pl,
+                                           status=dw.status)
+        assert_close(bf16_to_f64(out_s), ref, what=f"verify T={T} chunk {chunk}")
+    # the last query token sees the whole sequence: same as plain decode attention (up to rounding)
+    plain = pda.paged_decode_attention(dq[:, -1].contiguous(), dw.k_cache, dw.v_cache, dw.block_table,
+                                       dw.seq_lens, float(w.scale), status=dw.status)
+    assert np.abs(bf16_to_f64(plain) - bf16_to_f64(out)[:, -1]).max() < 1e-2
+    assert int(dw.status.item()) == 0
+
+
+def test_verify_attention_fp8_and_causal_needle(oracle):
+    w = W.prefix_fp8(seed=46, batch=4)
+    T = 16
+    q, _, _ = verify_inputs(w, T, 21)
+    ref, _ = oracle.paged_verify_attention(q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.scale,
+                                           w.k_scale, w.v_scale)
+    dw = DeviceWorkload(w)
+    out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                     float(w.scale), k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+    assert_close(bf16_to_f64(out), ref, "e4m3", what="verify fp8")
+    assert int(dw.status.item()) == 0
+
+    # causal structure: make the LAST key of a block dominant for every query; only the last
+    # query may see it, every earlier one must not
+    lens = [200]
+    w = W.make_workload("needle", lens, 4, 1, 128, seed=23)
+    q, kn, vn = verify_inputs(w, T, 24)
+    q[:] = q[:, :1, :1]                       # one q row everywhere
+    qf = W.bf16_bits_to_f32(q[0, 0, 0]).astype(np.float64)
+    kn[0, -1, 0] = W.f32_to_bf16_bits((40.0 / (float(w.scale) * (qf @ qf)) * qf).astype(np.float32))
+    vn[0, -1, 0] = W.f32_to_bf16_bits(np.arange(1, 129, dtype=np.float32))
+    dw = DeviceWorkload(w)
+    pda.kv_append_tokens(bf16_tensor(kn), bf16_tensor(vn), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens)
+    out = bf16_to_f64(pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table,
+                                                 dw.seq_lens, float(w.scale)))
+    assert np.abs(out[0, -1, 0] - np.arange(1, 129)).max() <= 0.5
+    assert np.abs(out[0, :-1]).max() < 3.0    # N(0,1) averages, nowhere near 1..128
+
+
+@pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
+@pytest.mark.parametrize("B", [3, 40])
+def test_shared_prefix_cascade(oracle, kv_dtype, B):
+    rng = np.random.default_rng(7)
+    prefix = 512
+    lens = prefix + rng.integers(0, 300, size=B)
+    lens[0] = prefix                        # a sequence with an empty suffix
+    w = W.make_workload("cascade", lens, 32, 8, 128, kv_dtype=kv_dtype, seed=29, shared_prefix_tokens=prefix)
+    assert (w.block_table[:, :prefix // 16] == w.block_table[0, :prefix // 16]).all()
+    dw = DeviceWorkload(w)
+    if kv_dtype == "bf16":
+        dw.append()
+    from util import host_appended
+    k, v = host_appended(oracle, w)
+    ref = oracle_out(oracle, w, k, v)
+    for pchunk, chunk in ((128, 64), (512, 256)):
+        mc = (prefix + pchunk - 1) // pchunk + pda.max_chunks(int(lens.max()) - prefix + 1, chunk)
+        po = torch.full((B, 32, mc, 128), float("nan"), dtype=torch.float32, device="cuda")
+        pl = torch.full((B, 32, mc), float("nan"), dtype=torch.float32, device="cuda")
+        out = pda.paged_prefix_decode_attention(dw.q, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                                float(w.scale), prefix, pchunk, chunk, po, pl,
+                                                k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+        assert_close(bf16_to_f64(out), ref, kv_dtype, what=f"cascade {kv_dtype} B={B} chunks {pchunk}/{chunk}")
+    plain = dw.attend()
+    assert np.abs(bf16_to_f64(plain) - bf16_to_f64(out)).max() < 2e-2
+    assert int(dw.status.item()) == 0

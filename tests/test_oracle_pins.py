@@ -378,3 +378,58 @@ def test_window_matches_library_sdpa_on_the_last_tokens(oracle, window):
     out2, lse2 = oracle.paged_decode_reduce(po, pl, w.seq_lens, 32)
     np.testing.assert_allclose(out2, out, rtol=0, atol=1e-12)
     np.testing.assert_allclose(lse2, lse, rtol=0, atol=1e-12)
+
+
+# ---- multi-token append and verification (causal block) attention -------------------------
+
+def verify_case(oracle, lens, T, Hq, Hkv, D, seed):
+    """A workload whose last T tokens per sequence are appended as a block; returns the pieces."""
+    w = W.make_workload("verify", lens, Hq, Hkv, D, seed=seed)
+    rng = np.random.default_rng(seed + 1)
+    B = len(lens)
+    q = W.f32_to_bf16_bits(rng.standard_normal((B, T, Hq, D), dtype=np.float32))
+    kn = W.f32_to_bf16_bits(rng.standard_normal((B, T, Hkv, D), dtype=np.float32))
+    vn = W.f32_to_bf16_bits(rng.standard_normal((B, T, Hkv, D), dtype=np.float32))
+    k, v = w.k_cache.copy(), w.v_cache.copy()
+    oracle.kv_append_tokens(kn, vn, k, v, w.block_table, w.seq_lens)
+    return w, q, kn, vn, k, v
+
+
+def test_multi_token_append_places_each_token(oracle):
+    w, q, kn, vn, k, v = verify_case(oracle, [16, 17, 40, 100], 16, 8, 2, 64, seed=3)
+    expect_k, expect_v = w.k_cache.copy(), w.v_cache.copy()
+    for b, L in enumerate([16, 17, 40, 100]):
+        for i in range(16):
+            pos = L - 16 + i
+            page = w.block_table[b, pos // 16]
+            expect_k[page, :, pos % 16, :] = kn[b, i]
+            expect_v[page, :, pos % 16, :] = vn[b, i]
+    assert (k == expect_k).all() and (v == expect_v).all()
+    # one token per sequence is the single-token append
+    k1, v1 = w.k_cache.copy(), w.v_cache.copy()
+    k2, v2 = w.k_cache.copy(), w.v_cache.copy()
+    oracle.kv_append(w.k_new, w.v_new, k1, v1, w.block_table, w.seq_lens)
+    oracle.kv_append_tokens(w.k_new[:, None], w.v_new[:, None], k2, v2, w.block_table, w.seq_lens)
+    assert (k1 == k2).all() and (v1 == v2).all()
+
+
+@pytest.mark.parametrize("T", [1, 4, 16])
+def test_verify_attention_matches_library_sdpa_with_causal_mask(oracle, T):
+    lens = [16, 17, 40, 100]
+    w, q, kn, vn, k, v = verify_case(oracle, lens, T, 8, 2, 64, seed=9)
+    out, lse = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
+    G = 4
+    for b, L in enumerate(lens):
+        K, V = dense_kv(w, k, v, b)
+        qq = torch.from_numpy(W.bf16_bits_to_f32(q[b]).astype(np.float64)).permute(1, 0, 2)[None]  # [1,Hq,T,D]
+        Kt = torch.from_numpy(K).repeat_interleave(G, dim=0)[None]
+        Vt = torch.from_numpy(V).repeat_interleave(G, dim=0)[None]
+        mask = torch.arange(L)[None, :] <= (L - T + torch.arange(T))[:, None]               # [T, L]
+        o = torch.nn.functional.scaled_dot_product_attention(qq, Kt, Vt, attn_mask=mask, scale=float(w.scale))
+        np.testing.assert_allclose(out[b], o[0].permute(1, 0, 2).numpy(), rtol=0, atol=1e-12)
+    # the last query token sees everything: it equals plain decode attention with that q
+    full, lse_full = oracle.paged_decode_attention(q[:, -1], k, v, w.block_table, w.seq_lens, w.scale)
+    assert (out[:, -1] == full).all() and (lse[:, -1] == lse_full).all()
+    # the first query token of a block that starts the sequence sees only itself: out = its V row
+    if T == 16:
+        assert (out[0, 0, 0] == W.bf16_bits_to_f32(vn[0, 0, 0]).astype(np.float64)).all()
