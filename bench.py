@@ -32,7 +32,10 @@ METRIC = "paged decode attention KV GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # chunk_tokens each workload is timed with (longctx is fixed by its definition)
-DEFAULT_CHUNK = {"tiny": 0, "llama8b": 0, "longctx": 2048, "chat70b": 0, "prefix_fp8": 0}
+DEFAULT_CHUNK = {"tiny": 0, "llama8b": 0, "longctx": 2048, "chat70b": 0, "prefix_fp8": 0,
+                 "scenario_c": 2048}
+# shared prefix length of the workloads that have one (for --mode cascade)
+PREFIX_TOKENS = {"prefix_fp8": 2048, "scenario_c": 32768}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu
 # capture summarised under profiles/ (None: not captured for that workload)
 NCU_TRAFFIC_BYTES = {"llama8b": 621_190_000}  # profiles/attention_tma_llama8b_ncu.md
@@ -210,7 +213,49 @@ def run_gpu(args):
     flags = {"tma": 0, "generic": pda.PDA_FLAG_FORCE_GENERIC}[args.kernel]
     launches_per_step = 1 if fused else (1 if k_new is not None else 0) + 1 + (1 if chunk else 0)
 
+    mode = args.mode
+    if mode == "cascade":
+        prefix = PREFIX_TOKENS[w.name]
+        pchunk, schunk = args.prefix_chunk, (chunk or 256)
+        mc = (prefix + pchunk - 1) // pchunk + pda.max_chunks(int(w.seq_lens.max()) - prefix + 1, schunk)
+        part_o = torch.empty((w.batch, w.num_q_heads, mc, w.head_dim), dtype=torch.float32, device=dev)
+        part_lse = torch.empty((w.batch, w.num_q_heads, mc), dtype=torch.float32, device=dev)
+        launches_per_step = 3 + (1 if k_new is not None else 0)
+    if mode == "verify":
+        T = args.verify_tokens
+        g = torch.Generator(device=dev).manual_seed(1)
+        vq = torch.randn((w.batch, T, w.num_q_heads, w.head_dim), generator=g, device=dev).to(torch.bfloat16)
+        vk = torch.randn((w.batch, T, w.num_kv_heads, w.head_dim), generator=g, device=dev).to(torch.bfloat16)
+        vv = torch.randn((w.batch, T, w.num_kv_heads, w.head_dim), generator=g, device=dev).to(torch.bfloat16)
+        vout = torch.empty_like(vq)
+        vpo = vpl = None
+        if chunk:
+            mc = pda.max_chunks(int(w.seq_lens.max()), chunk)
+            vpo = torch.empty((w.batch, T, w.num_q_heads, mc, w.head_dim), dtype=torch.float32, device=dev)
+            vpl = torch.empty((w.batch, T, w.num_q_heads, mc), dtype=torch.float32, device=dev)
+        launches_per_step = 2 + (1 if chunk else 0)
+
     def step(ev=None):
+        if mode == "cascade":
+            if k_new is not None:
+                pda.kv_append(k_new, v_new, k_cache, v_cache, bt, sl, status=status)
+            if ev:
+                ev[0].record(stream)
+            pda.paged_prefix_decode_attention(q, k_cache, v_cache, bt, sl, float(w.scale), prefix, pchunk,
+                                              schunk, part_o, part_lse, out=out, k_scale=k_scale,
+                                              v_scale=v_scale, status=status)
+            if ev:
+                ev[1].record(stream)
+            return
+        if mode == "verify":
+            pda.kv_append_tokens(vk, vv, k_cache, v_cache, bt, sl, status=status)
+            if ev:
+                ev[0].record(stream)
+            pda.paged_verify_attention(vq, k_cache, v_cache, bt, sl, float(w.scale), chunk_tokens=chunk,
+                                       out=vout, part_o=vpo, part_lse=vpl, status=status)
+            if ev:
+                ev[1].record(stream)
+            return
         if fused:   # append + attention + reduce in one launch
             if ev:
                 ev[0].record(stream)
@@ -279,7 +324,7 @@ def run_gpu(args):
 
     # ---- end to end from pinned host buffers (bf16 workloads) --------------------------------
     e2e = None
-    if k_new is not None:
+    if k_new is not None and mode == "decode":
         pin = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
         hq, hk, hv, hbt, hsl = pin(w.q), pin(w.k_new), pin(w.v_new), pin(w.block_table), pin(w.seq_lens)
         dq, dk, dv = torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new)
@@ -321,7 +366,7 @@ def run_gpu(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.kv_dtype == "bf16" else "e4m3",
             "data": "synthetic", "config": config_of(w, chunk, world),
             "tokens_per_s": batch_all / (ms_step * 1e-3),
-            "path": f"{args.path}/{args.kernel}",
+            "path": f"{args.path}/{args.kernel}" if mode == "decode" else mode,
             "pct_of_nominal_hbm_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
             "attention_ms": ms_attn,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -361,6 +406,11 @@ def main():
     ap.add_argument("--chunk", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
+    ap.add_argument("--mode", default="decode", choices=["decode", "cascade", "verify"],
+                    help="cascade: paged_prefix_decode_attention on a shared-prefix workload; "
+                         "verify: kv_append_tokens + paged_verify_attention with --verify-tokens queries")
+    ap.add_argument("--prefix-chunk", type=int, default=512)
+    ap.add_argument("--verify-tokens", type=int, default=16)
     ap.add_argument("--path", default="fused", choices=["fused", "separate"],
                     help="fused: one paged_decode_step launch; separate: kv_append, attention, reduce")
     ap.add_argument("--kernel", default="tma", choices=["tma", "generic"],

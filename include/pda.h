@@ -170,6 +170,22 @@ int kv_append_tokens(const void* k_new, const void* v_new, void* k_cache, void* 
                      int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
                      int32_t n_new, int32_t* status, pda_stream_t stream);
 
+/* Quantising KV append into e4m3 caches (no counterpart in the paper, whose one
+ * remark on KV quantisation is negative; this is the library's policy). k_new,
+ * v_new: [batch, num_kv_heads, head_dim] bf16. For K and V separately and every kv
+ * head, with slot = (L-1) % page_size of the target page:
+ *   slot == 0: scale[page, head] = amax(row) * 2 / 448 (1 if the row is all zero)
+ *              is stored -- the page's scale is fixed by its first row;
+ *   slot  > 0: the stored scale is reused;
+ *   bytes = e4m3(row / scale): IEEE fp32 division, round to nearest even,
+ *           saturating at +-448.
+ * k_scale, v_scale: [num_pages, num_kv_heads] fp32, read and written. head_dim must
+ * be a multiple of 64. Target slots must be distinct across the batch. */
+int kv_append_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                  const pda_cache_desc* desc, float* k_scale, float* v_scale,
+                  const int32_t* block_table, int32_t block_table_stride,
+                  const int32_t* seq_lens, int32_t batch, int32_t* status, pda_stream_t stream);
+
 /* Verification attention over a block of n_query_tokens draft tokens per sequence
  * (the predicted-output verifier of the paper scores 16-token blocks in one pass:
  * Section 4.2 and Appendix A, Scenario B; the paper prints no formula -- this is

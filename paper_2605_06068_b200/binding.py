@@ -23,7 +23,7 @@ EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
            "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
            "paged_decode_step", "pda_advance_seq_lens", "paged_window_decode_attention", "kv_append_tokens",
-           "paged_verify_attention", "paged_prefix_decode_attention"]
+           "paged_verify_attention", "paged_prefix_decode_attention", "kv_append_fp8"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
@@ -57,6 +57,7 @@ def lib():
         L.paged_decode_step_host.argtypes = [vp] * 5 + [vp] * 5 + [vp, vp, dp, i32, i32, i32, f32,
                                                                  i32, vp, vp, i32, vp, vp, vp, vp, vp]
         L.pda_workspace_ints.argtypes = [i32, i32]
+        L.kv_append_fp8.argtypes = [vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, vp, vp]
         L.kv_append_tokens.argtypes = [vp, vp, vp, vp, dp, vp, i32, vp, i32, i32, vp, vp]
         L.paged_verify_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, i32, f32,
                                              i32, vp, vp, vp, i32, vp, vp]
@@ -308,3 +309,14 @@ def paged_prefix_decode_attention(q, k_cache, v_cache, block_table, seq_lens, sc
         _ptr(part_lse), mc, _ptr(status), _stream(stream))
     _check(rc, "paged_prefix_decode_attention")
     return out
+
+
+def kv_append_fp8(k_new, v_new, k_cache, v_cache, k_scale, v_scale, block_table, seq_lens,
+                  status=None, stream=None):
+    """Quantising append of bf16 rows into e4m3 caches (scale fixed by each page's first row)."""
+    desc = cache_desc(k_cache)
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_scale.is_contiguous()
+    rc = lib().kv_append_fp8(_ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), C.byref(desc),
+                             _ptr(k_scale), _ptr(v_scale), _ptr(block_table), block_table.stride(0),
+                             _ptr(seq_lens), seq_lens.shape[0], _ptr(status), _stream(stream))
+    _check(rc, "kv_append_fp8")

@@ -260,5 +260,14 @@ def prefix_fp8(seed=BASE_SEED + 4, batch=128) -> Workload:
                          shared_prefix_tokens=2048)
 
 
+def scenario_c(seed=BASE_SEED + 5, batch=20) -> Workload:
+    """Shared-prefix prompt caching shaped like the paper's Scenario C: 20 concurrent
+    sequences, one 32768-token shared prefix plus a private suffix of 128..256 tokens
+    (its 128-token suffix plus up to 128 generated tokens), 32 q / 8 kv heads, head_dim 128."""
+    rng = np.random.default_rng(np.random.PCG64(seed))
+    L = 32768 + rng.integers(128, 256, size=batch, endpoint=True)
+    return make_workload("scenario_c", L, 32, 8, 128, seed=seed, rng=rng, shared_prefix_tokens=32768)
+
+
 WORKLOADS = {"tiny": tiny, "llama8b": llama8b, "longctx": longctx, "chat70b": chat70b,
-             "prefix_fp8": prefix_fp8}
+             "prefix_fp8": prefix_fp8, "scenario_c": scenario_c}

@@ -466,3 +466,45 @@ def test_sliding_window(oracle, flags, shape):
             out_s = pda.paged_decode_reduce(po, pl, dw.seq_lens, chunk)
             assert_close(bf16_to_f64(out_s), ref, what=f"window {window} chunk {chunk}")
     assert status_of(dw) == 0
+
+
+# ---- quantising append into e4m3 caches ------------------------------------------------------
+
+@pytest.mark.parametrize("shape", [(8, 2, 64), (32, 8, 128)])
+def test_fp8_append_bit_exact_and_attention_on_the_grown_cache(oracle, shape):
+    Hq, Hkv, D = shape
+    B, T = 5, 40
+    start = np.array([0, 3, 15, 16, 31], np.int32)
+    rng = np.random.default_rng(11)
+    pages_per_seq = (int(start.max()) + T + 15) // 16
+    n_pages = B * pages_per_seq + 3
+    table = rng.permutation(n_pages)[:B * pages_per_seq].reshape(B, pages_per_seq).astype(np.int32)
+    hk = np.full((n_pages, Hkv, 16, D), 0xFF, np.uint8); hv = hk.copy()
+    hks = np.full((n_pages, Hkv), np.nan, np.float32); hvs = hks.copy()
+    # caches start empty except for `start` tokens appended through the oracle itself
+    dk, dv = torch.from_numpy(hk.copy()).cuda(), torch.from_numpy(hv.copy()).cuda()
+    dks, dvs = torch.from_numpy(hks.copy()).cuda(), torch.from_numpy(hvs.copy()).cuda()
+    bt = torch.from_numpy(table).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lens = np.zeros(B, np.int32)
+    for t in range(int(start.max()) + T):
+        active = (t < start + T)
+        lens = lens + active.astype(np.int32)
+        cur = np.where(active, lens, 0).astype(np.int32)      # inactive rows append nothing
+        scale_up = 1.0 + 5.0 * (t % 7 == 3)                     # some rows exceed their page's range
+        kn = W.f32_to_bf16_bits((rng.standard_normal((B, Hkv, D)) * scale_up).astype(np.float32))
+        vn = W.f32_to_bf16_bits(rng.standard_normal((B, Hkv, D)).astype(np.float32))
+        oracle.kv_append_e4m3(kn, vn, hk, hv, hks, hvs, table, cur)
+        pda.kv_append_fp8(bf16_tensor(kn), bf16_tensor(vn), dk, dv, dks, dvs, bt,
+                          torch.from_numpy(cur).cuda(), status=status)
+    assert (dk.cpu().numpy() == hk).all() and (dv.cpu().numpy() == hv).all()
+    gks, gvs = dks.cpu().numpy(), dvs.cpu().numpy()
+    live = ~np.isnan(hks)
+    assert (np.isnan(gks) == np.isnan(hks)).all() and (gks[live] == hks[live]).all() and (gvs[live] == hvs[live]).all()
+    assert int(status.item()) == 0
+    # attention over the grown cache
+    q = W.f32_to_bf16_bits(rng.standard_normal((B, Hq, D), dtype=np.float32))
+    ref, _ = oracle.paged_decode_attention(q, hk, hv, table, lens, np.float32(1 / np.sqrt(D)), hks, hvs)
+    out = pda.paged_decode_attention(bf16_tensor(q), dk, dv, bt, torch.from_numpy(lens).cuda(),
+                                     float(np.float32(1 / np.sqrt(D))), k_scale=dks, v_scale=dvs, status=status)
+    assert_close(bf16_to_f64(out), ref, "e4m3", what="attention after fp8 appends")

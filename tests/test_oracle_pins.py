@@ -433,3 +433,45 @@ def test_verify_attention_matches_library_sdpa_with_causal_mask(oracle, T):
     # the first query token of a block that starts the sequence sees only itself: out = its V row
     if T == 16:
         assert (out[0, 0, 0] == W.bf16_bits_to_f32(vn[0, 0, 0]).astype(np.float64)).all()
+
+
+# ---- quantising append ---------------------------------------------------------------------
+
+def test_e4m3_append_policy_against_library_cast(oracle):
+    """Scale is set by the page's first row (amax*2/448); later rows reuse it and saturate."""
+    rng = np.random.default_rng(3)
+    Hkv, D, P = 2, 64, 16
+    n_pages = 4
+    kc = np.full((n_pages, Hkv, P, D), 0xFF, np.uint8); vc = kc.copy()
+    ks = np.full((n_pages, Hkv), np.nan, np.float32); vs = ks.copy()
+    table = np.array([[2, 0], [3, 1]], np.int32)
+    hist = {}
+    for step in range(20):                       # lengths 1..20: pages opened at L=1 and L=17
+        lens = np.array([step + 1, step + 1], np.int32)
+        kn = W.f32_to_bf16_bits((rng.standard_normal((2, Hkv, D)) * (1 + 3 * (step % 5 == 4))).astype(np.float32))
+        vn = W.f32_to_bf16_bits(rng.standard_normal((2, Hkv, D)).astype(np.float32))
+        if step == 7:
+            kn[0, 0] = 0                          # an all-zero row
+        oracle.kv_append_e4m3(kn, vn, kc, vc, ks, vs, table, lens)
+        hist[step] = (kn, vn)
+    # restate with torch's cast (saturating by clamp) page by page
+    for b in range(2):
+        for step in range(20):
+            page, slot = table[b, step // 16], step % 16
+            first = hist[(step // 16) * 16]
+            for g in range(Hkv):
+                for src, cache, scales in ((0, kc, ks), (1, vc, vs)):
+                    x0 = torch.from_numpy(W.bf16_bits_to_f32(first[src][b, g]))
+                    sc = (x0.abs().max() * 2.0) / 448.0
+                    assert scales[page, g] == np.float32(sc)
+                    x = torch.from_numpy(W.bf16_bits_to_f32(hist[step][src][b, g]))
+                    y = (x / sc).clamp(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+                    got = cache[page, g, slot]
+                    same = (got == y) | ((got & 0x7F) == 0) & ((y & 0x7F) == 0)   # +-0 alike
+                    assert same.all(), (b, step, g, src)
+    # untouched slots keep their fill; the zero row quantises to zero codes
+    assert (kc[table[0, 1], :, 4:, :] == 0xFF).all()
+    assert ((kc[table[0, 0], 0, 7] & 0x7F) == 0).all()
+    # a row 4x larger than the page's first row saturates at +-448 somewhere
+    t = oracle.e4m3_decode_table()
+    assert np.abs(t[kc[table[0, 0], :, 4]]).max() == 448.0
