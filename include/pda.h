@@ -64,6 +64,9 @@ extern "C" {
 #define PDA_FLAG_FORCE_GENERIC 1u /* use the plain CUDA-core kernel even where the
                                      TMA + tensor-core kernel applies (for testing) */
 
+#define PDA_FLAG_MQ_MMA_SYNC 2u   /* multi-query calls (verify, shared prefix): use the mma.sync
+                                     kernel even where the tcgen05 + TMEM kernel applies */
+
 typedef void* pda_stream_t; /* cudaStream_t */
 
 /* Describes k_cache and v_cache (both have the same geometry).
@@ -199,14 +202,17 @@ int kv_append_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_c
  *             inside this call.  `out` is always written.
  * The query rows of a kv head's group form dense tensor-core tiles (rows = tokens x
  * group size), so each page is fetched once per block, not once per token.
- * Supported: head_dim 64 or 128 (bf16), 128 (e4m3). */
+ * bf16 KV with head_dim 128 runs on tcgen05 tensor-core tiles with the accumulators
+ * in tensor memory (128 query rows per CTA); other supported shapes (head_dim 64
+ * bf16, 128 e4m3) and PDA_FLAG_MQ_MMA_SYNC use the mma.sync kernel. */
 int paged_verify_attention(const void* q, const void* k_cache, const void* v_cache,
                            const pda_cache_desc* desc, const float* k_scale,
                            const float* v_scale, const int32_t* block_table,
                            int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
                            int32_t num_q_heads, int32_t n_query_tokens, float scale,
                            int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
-                           int32_t max_chunks, int32_t* status, pda_stream_t stream);
+                           int32_t max_chunks, uint32_t flags, int32_t* status,
+                           pda_stream_t stream);
 
 /* Decode attention for a batch whose sequences all start with the SAME
  * prefix_tokens tokens stored in the same physical pages (the shared-prefix
@@ -233,7 +239,8 @@ int paged_prefix_decode_attention(const void* q, const void* k_cache, const void
                                   int32_t batch, int32_t num_q_heads, float scale,
                                   int32_t prefix_tokens, int32_t prefix_chunk_tokens,
                                   int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
-                                  int32_t max_chunks, int32_t* status, pda_stream_t stream);
+                                  int32_t max_chunks, uint32_t flags, int32_t* status,
+                                  pda_stream_t stream);
 
 /* Merge of split-KV partials (the reduce step of flash-decoding; exact algebra):
  *     out[b,h,:] = sum_c w_c part_o[b,h,c,:] / sum_c w_c,

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libpda.so")
 
 PDA_BF16, PDA_FP8_E4M3 = 0, 1
 PDA_FLAG_FORCE_GENERIC = 1
+PDA_FLAG_MQ_MMA_SYNC = 2
 DEV_STATUS = {0: "ok", 1: "bad page id", 2: "seq_len exceeds block table", 3: "copy wait timed out"}
 
 EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
@@ -60,9 +61,9 @@ def lib():
         L.kv_append_fp8.argtypes = [vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, vp, vp]
         L.kv_append_tokens.argtypes = [vp, vp, vp, vp, dp, vp, i32, vp, i32, i32, vp, vp]
         L.paged_verify_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, i32, f32,
-                                             i32, vp, vp, vp, i32, vp, vp]
+                                             i32, vp, vp, vp, i32, u32, vp, vp]
         L.paged_prefix_decode_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
-                                                    i32, i32, i32, vp, vp, vp, i32, vp, vp]
+                                                    i32, i32, i32, vp, vp, vp, i32, u32, vp, vp]
         L.paged_window_decode_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
                                                     i32, i32, vp, vp, vp, i32, u32, vp, vp]
         L.pda_advance_seq_lens.argtypes = [vp, i32, i32, vp]
@@ -272,7 +273,7 @@ def kv_append_tokens(k_new, v_new, k_cache, v_cache, block_table, seq_lens, stat
 
 
 def paged_verify_attention(q, k_cache, v_cache, block_table, seq_lens, scale, chunk_tokens=0, out=None,
-                           part_o=None, part_lse=None, k_scale=None, v_scale=None, status=None,
+                           part_o=None, part_lse=None, k_scale=None, v_scale=None, flags=0, status=None,
                            stream=None):
     """Causal attention of a block of query tokens ``q [B,T,Hq,D]``; returns ``out [B,T,Hq,D]``."""
     desc = cache_desc(k_cache)
@@ -287,14 +288,15 @@ def paged_verify_attention(q, k_cache, v_cache, block_table, seq_lens, scale, ch
     rc = lib().paged_verify_attention(
         _ptr(q), _ptr(k_cache), _ptr(v_cache), C.byref(desc), _ptr(k_scale), _ptr(v_scale),
         _ptr(block_table), block_table.stride(0), _ptr(seq_lens), B, Hq, T, float(scale),
-        chunk_tokens, _ptr(out), _ptr(part_o), _ptr(part_lse), mc, _ptr(status), _stream(stream))
+        chunk_tokens, _ptr(out), _ptr(part_o), _ptr(part_lse), mc, flags, _ptr(status),
+        _stream(stream))
     _check(rc, "paged_verify_attention")
     return out
 
 
 def paged_prefix_decode_attention(q, k_cache, v_cache, block_table, seq_lens, scale, prefix_tokens,
                                   prefix_chunk_tokens, chunk_tokens, part_o, part_lse, out=None,
-                                  k_scale=None, v_scale=None, status=None, stream=None):
+                                  k_scale=None, v_scale=None, flags=0, status=None, stream=None):
     """Decode attention of a batch sharing its first ``prefix_tokens`` tokens' pages."""
     desc = cache_desc(k_cache)
     B, Hq, D = q.shape
@@ -306,7 +308,7 @@ def paged_prefix_decode_attention(q, k_cache, v_cache, block_table, seq_lens, sc
         _ptr(q), _ptr(k_cache), _ptr(v_cache), C.byref(desc), _ptr(k_scale), _ptr(v_scale),
         _ptr(block_table), block_table.stride(0), _ptr(seq_lens), B, Hq, float(scale),
         int(prefix_tokens), int(prefix_chunk_tokens), int(chunk_tokens), _ptr(out), _ptr(part_o),
-        _ptr(part_lse), mc, _ptr(status), _stream(stream))
+        _ptr(part_lse), mc, flags, _ptr(status), _stream(stream))
     _check(rc, "paged_prefix_decode_attention")
     return out
 

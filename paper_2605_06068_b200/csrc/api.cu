@@ -220,7 +220,8 @@ int paged_verify_attention(const void* q, const void* k_cache, const void* v_cac
                            int32_t block_table_stride, const int32_t* seq_lens, int32_t batch,
                            int32_t num_q_heads, int32_t n_query_tokens, float scale,
                            int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
-                           int32_t max_chunks, int32_t* status, pda_stream_t stream) {
+                           int32_t max_chunks, uint32_t flags, int32_t* status,
+                           pda_stream_t stream) {
   AttnParams p;
   if (n_query_tokens <= 0 || n_query_tokens > 4096) return PDA_ERR_INVALID_ARG;
   if (!out && batch > 0) return PDA_ERR_INVALID_ARG;
@@ -234,9 +235,13 @@ int paged_verify_attention(const void* q, const void* k_cache, const void* v_cac
   p.scale = scale;
   p.out = static_cast<__nv_bfloat16*>(out);
   pda::MqParams mp{p, n_query_tokens, 1, 0, max_chunks};
-  if (!pda::attention_mq_supports(mp)) return PDA_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cudaError_t e = pda::launch_attention_mq(mp, s)) return static_cast<int>(e);
+  if (!(flags & PDA_FLAG_MQ_MMA_SYNC) && pda::attention_mq_tc_supports(mp)) {
+    if (cudaError_t e = pda::launch_attention_mq_tc(mp, s)) return static_cast<int>(e);
+  } else {
+    if (!pda::attention_mq_supports(mp)) return PDA_ERR_UNSUPPORTED;
+    if (cudaError_t e = pda::launch_attention_mq(mp, s)) return static_cast<int>(e);
+  }
   if (chunk_tokens > 0)
     return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
                                                p.geom.head_dim, chunk_tokens, max_chunks, 0, 0,
@@ -251,7 +256,8 @@ int paged_prefix_decode_attention(const void* q, const void* k_cache, const void
                                   int32_t batch, int32_t num_q_heads, float scale,
                                   int32_t prefix_tokens, int32_t prefix_chunk_tokens,
                                   int32_t chunk_tokens, void* out, float* part_o, float* part_lse,
-                                  int32_t max_chunks, int32_t* status, pda_stream_t stream) {
+                                  int32_t max_chunks, uint32_t flags, int32_t* status,
+                                  pda_stream_t stream) {
   AttnParams p;
   if (prefix_tokens <= 0 || prefix_chunk_tokens <= 0 || chunk_tokens <= 0) return PDA_ERR_INVALID_ARG;
   if (prefix_tokens % pda::kPageSize || prefix_chunk_tokens % pda::kPageSize) return PDA_ERR_INVALID_ARG;
@@ -276,8 +282,13 @@ int paged_prefix_decode_attention(const void* q, const void* k_cache, const void
   pp.chunk_tokens = prefix_chunk_tokens;
   pp.chunk_slot0 = 0;
   pda::MqParams mp{pp, batch, 0, prefix_tokens, prefix_chunks};
-  if (!pda::attention_mq_supports(mp) || !pda::attention_tma_supports(p)) return PDA_ERR_UNSUPPORTED;
-  if (cudaError_t e = pda::launch_attention_mq(mp, s)) return static_cast<int>(e);
+  if (!pda::attention_tma_supports(p)) return PDA_ERR_UNSUPPORTED;
+  if (!(flags & PDA_FLAG_MQ_MMA_SYNC) && pda::attention_mq_tc_supports(mp)) {
+    if (cudaError_t e = pda::launch_attention_mq_tc(mp, s)) return static_cast<int>(e);
+  } else {
+    if (!pda::attention_mq_supports(mp)) return PDA_ERR_UNSUPPORTED;
+    if (cudaError_t e = pda::launch_attention_mq(mp, s)) return static_cast<int>(e);
+  }
   // (2) every sequence's own suffix, chunk slots after the prefix's
   AttnParams ps = p;
   ps.first_token = prefix_tokens;

@@ -1,0 +1,439 @@
+// Multi-query paged attention on the 5th-generation tensor cores (tcgen05 + TMEM),
+// bf16 KV, head_dim 128. Same contract as attention_mq.cu (verification of a
+// block of draft tokens; the shared-prefix part of a decode batch): up to 128
+// query rows (query tokens x group size) per CTA against one sequence's pages.
+//
+// This is the part of the path that is a real dense contraction, so it runs as
+// UMMA tiles with accumulators in tensor memory:
+//   S[128 x 64]  = Q[128 x D] . K^T     per 4 pages: per page 8 tcgen05.mma of
+//                                        M128 x N16 x K16 (K-major A and B)
+//   O[128 x D]  += P[128 x 64] . V      per page 1 tcgen05.mma M128 x N128 x K16
+//                                        (A = P from shared memory, B = V MN-major)
+// The (page, head) tiles land through the same 5-D TMA map as everywhere else:
+// [128-byte line][16 slots][128 B] with the 128-byte swizzle is already the
+// canonical UMMA layout, K-major for K (rows = tokens, contraction over d) and
+// MN-major for V (contraction over the 16 tokens of the page), so no data is
+// rearranged in shared memory.
+//
+// Warp roles (6 warps): 0-3 softmax (thread t <-> TMEM lane t <-> query row t),
+// 4 TMA producer, 5 MMA issue + TMEM allocation. Per iteration of 64 tokens:
+//   MMA warp:   wait stage -> S MMAs -> commit(bar_s) ; wait bar_p -> PV MMAs ->
+//               commit(stage empty), commit(bar_o)
+//   softmax:    wait bar_s -> tcgen05.ld S -> scale, mask, row max (thread-local)
+//               -> wait bar_o of the previous iteration -> (rarely) rescale O in
+//               TMEM when the running max grew by more than 2^8 -> P = exp2(..)
+//               as bf16 into the swizzled P tile -> arrive(bar_p)
+// All mbarrier waits are bounded; TMEM is always released before the CTA exits.
+#include "common.cuh"
+#include "tma_ptx.cuh"
+
+namespace pda {
+
+namespace {
+
+constexpr int kTcD = 128;               // head_dim
+constexpr int kTcRows = 128;            // query rows per CTA (UMMA M)
+constexpr int kTcPagesPerIter = 4;      // 64 tokens per iteration
+constexpr int kTcStages = 4;
+constexpr int kTcTileBytes = kPageSize * kTcD * 2;        // 4096: one K or V page tile
+constexpr int kTcPageBytes = 2 * kTcTileBytes;            // K then V
+constexpr int kTcStageBytes = kTcPagesPerIter * kTcPageBytes;  // 32 KB
+constexpr int kTcQBytes = kTcRows * kTcD * 2;             // 32 KB: [2 lines][128 rows][128 B]
+constexpr int kTcPBytes = kTcRows * 128;                  // 16 KB: [128 rows][64 tokens] bf16
+constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcQBytes + kTcPBytes + 256 + 1024;
+constexpr int kTcThreads = 192;
+constexpr uint32_t kTmemCols = 256;     // S: columns 0..63, O: columns 64..191
+constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the max grows this much
+
+__device__ __forceinline__ void mbar_arrive_tc(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] . B[smem desc]; accumulate == 0 overwrites D
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field.
+__device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return static_cast<uint64_t>((smem_addr >> 4) & 0x3FFFu) |
+         (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: f32 accumulate, bf16 A and B, A K-major, M = 128.
+__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+         (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTcRows >> 4) << 24);
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
+                       const __grid_constant__ CUtensorMap v_map, MqParams mp) {
+  const AttnParams& p = mp.a;
+  constexpr int D = kTcD;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_smem = smem + kTcStages * kTcStageBytes;
+  uint8_t* p_smem = q_smem + kTcQBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(p_smem + kTcPBytes);  // full[4], empty[4], s, p, o
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 3);
+  int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = p.group, T = mp.n_q;
+  const int rows_total = T * G;
+  const int n_rb = (rows_total + kTcRows - 1) / kTcRows;
+  const int c = blockIdx.x, g = blockIdx.y / n_rb, rb = blockIdx.y % n_rb, b = blockIdx.z;
+  const bool split = p.chunk_tokens > 0;
+
+  const int L = mp.kv_len_fixed > 0 ? mp.kv_len_fixed : max(p.seq_lens[b], 0);
+  int t0 = p.first_token, t1 = L;
+  if (split) {
+    t0 = p.first_token + c * p.chunk_tokens;
+    if (t0 >= L) return;
+    t1 = min(t0 + p.chunk_tokens, L);
+  }
+  // once any CTA of this launch has reported a timed-out wait, the rest do not start
+  if (p.status != nullptr && *reinterpret_cast<volatile int32_t*>(p.status) == PDA_DEV_TIMEOUT) return;
+  int err = 0;
+  if (static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
+      (split && static_cast<int64_t>(L - p.first_token) >
+                    static_cast<int64_t>(p.max_chunks - p.chunk_slot0) * p.chunk_tokens))
+    err = PDA_DEV_BAD_SEQ_LEN;
+  const int page0 = t0 / kPageSize;
+  const int n_pages = err ? 0 : (t1 + kPageSize - 1) / kPageSize - page0;
+  const int n_iters = (n_pages + kTcPagesPerIter - 1) / kTcPagesPerIter;
+
+  const uint32_t ring = smem_u32(smem);
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
+  const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 8, bar_o = bar_p + 8;
+  if (tid == 0) {
+    for (int s = 0; s < kTcStages; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    mbar_init(bar_s, 1);
+    mbar_init(bar_p, 4);   // one arrival per softmax warp
+    mbar_init(bar_o, 1);
+    *cta_err = 0;
+    fence_mbar_init();
+    fence_proxy_async();
+  }
+  if (warp == 5) {  // tensor memory for S and O; this warp also releases it
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  // ---- Q tile: row r -> (query token r / G, head r % G), written in the swizzled K-major layout
+  if (warp < 4) {
+    const int r = rb * kTcRows + tid;
+    const bool valid = r < rows_total;
+    const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
+    const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
+#pragma unroll
+    for (int ch = 0; ch < 16; ++ch) {
+      const uint4 v = valid ? src[ch] : make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t dst = smem_u32(q_smem) + (ch >> 3) * (kTcRows * 128) + tid * 128 + (((ch & 7) ^ (tid & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+    }
+    fence_proxy_async();  // the tensor core reads this tile through the async proxy
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 64;
+
+  const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
+
+  if (warp == 4) {
+    // ================= TMA producer =================
+    bool bad = false;
+    int pg = 0;
+    for (int it = 0; it < n_iters; ++it) {
+      const int s = it % kTcStages;
+      if ((it & 7) == 0) {  // page ids of the next 8 iterations (32 pages), one per lane
+        pg = 0;
+        if (it * kTcPagesPerIter + lane < n_pages) {
+          const int v = table[page0 + it * kTcPagesPerIter + lane];
+          pg = (v < 0 || v >= p.geom.num_pages) ? -1 : v;
+        }
+      }
+      bool ok = true;
+      if (it >= kTcStages) ok = mbar_wait_bounded(empty0 + 8 * s, ((it / kTcStages) - 1) & 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
+      const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
+      if (lane == 0) mbar_expect_tx(full0 + 8 * s, n_here * kTcPageBytes);
+      for (int j = 0; j < n_here; ++j) {
+        const int page_raw = __shfl_sync(0xffffffffu, pg, (it & 7) * kTcPagesPerIter + j);
+        if (page_raw < 0) bad = true;
+        if (lane == 0) {
+          const uint32_t dst = ring + s * kTcStageBytes + j * kTcPageBytes;
+          tma_load_5d(dst, &k_map, full0 + 8 * s, 0, 0, 0, g, max(page_raw, 0));
+          tma_load_5d(dst + kTcTileBytes, &v_map, full0 + 8 * s, 0, 0, 0, g, max(page_raw, 0));
+        }
+      }
+    }
+    if (bad && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
+  } else if (warp == 5) {
+    // ================= MMA issue =================
+    constexpr uint32_t idesc_s = tc_idesc(16, false);
+    constexpr uint32_t idesc_pv = tc_idesc(D, true);
+    const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
+    for (int it = 0; it < n_iters; ++it) {
+      const int s = it % kTcStages;
+      bool ok = mbar_wait_bounded(full0 + 8 * s, (it / kTcStages) & 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
+      const uint32_t stage = ring + s * kTcStageBytes;
+      const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
+      // rows of the sequence's last page past its end may hold anything: clear them in V
+      const int tail = L - (page0 + it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
+      if (tail < kPageSize) {
+        const uint32_t vt = stage + (n_here - 1) * kTcPageBytes + kTcTileBytes;
+        for (int i = lane; i < (kPageSize - tail) * 16; i += 32) {
+          const int r = tail + i / 16, ch = i % 16;
+          asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_off(r, ch)), "r"(0));
+        }
+        fence_proxy_async();
+        __syncwarp();
+      }
+      tc_fence_after();
+      if (lane == 0) {
+        // S columns [16j, 16j+16) = Q . K_j^T, contraction over d in 8 steps of 16
+        for (int j = 0; j < n_here; ++j) {
+          const uint32_t kt = stage + j * kTcPageBytes;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint64_t a = tc_desc(q_addr + (ks >> 2) * (kTcRows * 128) + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = tc_desc(kt + (ks >> 2) * (kPageSize * 128) + (ks & 3) * 32, 16, 1024);
+            tc_mma(tmem_s + 16 * j, a, bd, idesc_s, ks > 0 ? 1u : 0u);
+          }
+        }
+        tc_commit(bar_s);
+      }
+      __syncwarp();
+      ok = mbar_wait_bounded(bar_p, it & 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
+      tc_fence_after();
+      if (lane == 0) {
+        // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page, V read MN-major
+        for (int j = 0; j < n_here; ++j) {
+          const uint32_t vt = stage + j * kTcPageBytes + kTcTileBytes;
+          const uint64_t a = tc_desc(p_addr + j * 32, 16, 1024);
+          const uint64_t bd = tc_desc(vt, kPageSize * 128, 1024);  // LBO: next 64 columns of d, SBO: next 8 tokens
+          tc_mma(tmem_o, a, bd, idesc_pv, (it > 0 || j > 0) ? 1u : 0u);
+        }
+        tc_commit(empty0 + 8 * s);  // the stage may be refilled once these MMAs have read it
+        tc_commit(bar_o);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ================= softmax: thread t owns query row t =================
+    const int r = rb * kTcRows + tid;
+    const int i_tok = r / G;
+    const int lim = mp.causal ? min(L, L - T + i_tok + 1) : L;
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;  // this warp's TMEM lanes
+    const float scale_log2 = p.scale * 1.4426950408889634f;
+    float m_ref = -INFINITY;   // reference max the accumulated O and l are scaled by
+    float l = 0.f;
+    bool alive = true;
+    for (int it = 0; it < n_iters && alive; ++it) {
+      bool ok = mbar_wait_bounded(bar_s, it & 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
+      tc_fence_after();
+      uint32_t sv[2][32];
+      tmem_ld32(tmem_s + lane_base, sv[0]);
+      tmem_ld32(tmem_s + lane_base + 32, sv[1]);
+      tmem_wait_ld();
+      const int tok0 = (page0 + it * kTcPagesPerIter) * kPageSize;
+      const int n_vis = min(lim, t1) - tok0;  // visible columns of this row in this iteration (may be <= 0)
+      float mx = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float x = __uint_as_float(sv[h][j]) * scale_log2;
+          x = (h * 32 + j < n_vis) ? x : -INFINITY;
+          sv[h][j] = __float_as_uint(x);
+          mx = fmaxf(mx, x);
+        }
+      // lazy rescaling: keep the old reference unless the max grew past the threshold
+      float m_new = m_ref;
+      if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = fmaxf(m_ref, mx);
+      const bool need = m_new != m_ref && m_ref != -INFINITY;
+      if (it > 0) {
+        ok = mbar_wait_bounded(bar_o, (it - 1) & 1);  // previous PV done: O is stable, P tile is free
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, need)) {
+          const float alpha = need ? ex2(m_ref - m_new) : 1.f;
+          l *= alpha;
+#pragma unroll
+          for (int cb = 0; cb < D / 32; ++cb) {
+            uint32_t ov[32];
+            tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
+            tmem_st32(tmem_o + lane_base + 32 * cb, ov);
+          }
+          tmem_wait_st();
+        }
+      }
+      m_ref = m_new;
+      const float ref = m_ref == -INFINITY ? 0.f : m_ref;
+      // P = exp2(S - ref) as bf16 into row `tid` of the swizzled [128 rows][128 B] tile
+      float lsum = 0.f;
+      const uint32_t prow = smem_u32(p_smem) + tid * 128;
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = ch * 8 + 2 * e;
+          const float p0 = ex2(__uint_as_float(sv[j >> 5][j & 31]) - ref);
+          const float p1 = ex2(__uint_as_float(sv[(j + 1) >> 5][(j + 1) & 31]) - ref);
+          lsum += p0 + p1;
+          w[e] = pack2<false>(p0, p1);
+        }
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};"
+                     ::"r"(prow + ((ch ^ (tid & 7)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]));
+      }
+      l += lsum;
+      fence_proxy_async();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_tc(bar_p);
+    }
+
+    // ---- finalise this row
+    bool ok = true;
+    if (alive && n_iters > 0) {
+      ok = mbar_wait_bounded(bar_o, (n_iters - 1) & 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
+      tc_fence_after();
+    }
+    // every softmax warp reaches this point together with its error view settled
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    const int dev_err = max(err, *cta_err);
+    if (dev_err && tid == 0) report(p.status, dev_err);
+    const bool valid_row = r < rows_total;
+    const bool live = !dev_err && alive && ok && l > 0.f;
+    const float inv = live ? 1.f / l : 0.f;
+    const int64_t qrow = (static_cast<int64_t>(b) * T + i_tok) * p.num_q_heads + g * G + (r % G);
+    constexpr float kLn2 = 0.6931471805599453f;
+#pragma unroll
+    for (int cb = 0; cb < D / 32; ++cb) {
+      uint32_t ov[32];
+      if (alive && ok && n_iters > 0) {  // warp-uniform
+        tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ov[j] = 0u;
+      }
+      if (valid_row) {
+        if (split) {
+          float4* dst = reinterpret_cast<float4*>(p.part_o + (qrow * p.max_chunks + p.chunk_slot0 + c) * D + 32 * cb);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            dst[j] = make_float4(live ? __uint_as_float(ov[4 * j]) * inv : 0.f, live ? __uint_as_float(ov[4 * j + 1]) * inv : 0.f,
+                                 live ? __uint_as_float(ov[4 * j + 2]) * inv : 0.f, live ? __uint_as_float(ov[4 * j + 3]) * inv : 0.f);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(p.out + qrow * D + 32 * cb);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              w[e] = pack2<false>(live ? __uint_as_float(ov[8 * j + 2 * e]) * inv : 0.f,
+                                  live ? __uint_as_float(ov[8 * j + 2 * e + 1]) * inv : 0.f);
+            dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+    if (split && valid_row)
+      p.part_lse[qrow * p.max_chunks + p.chunk_slot0 + c] = live ? (m_ref + __log2f(l)) * kLn2 : -INFINITY;
+  }
+
+  // ---- teardown: everyone is done with tensor memory before it is released
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace
+
+bool attention_mq_tc_supports(const MqParams& mp) {
+  const AttnParams& p = mp.a;
+  if (p.geom.dtype != PDA_BF16 || p.geom.head_dim != kTcD) return false;
+  if (p.group < 1 || mp.n_q < 1 || p.geom.num_pages < 1) return false;
+  const int64_t rows = static_cast<int64_t>(mp.n_q) * p.group;
+  return p.geom.num_kv_heads * ((rows + kTcRows - 1) / kTcRows) <= 65535;
+}
+
+cudaError_t launch_attention_mq_tc(const MqParams& mp, cudaStream_t stream) {
+  const AttnParams& p = mp.a;
+  alignas(64) CUtensorMap k_map, v_map;
+  if (!make_cache_tensor_map(&k_map, p.k_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
+                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2) ||
+      !make_cache_tensor_map(&v_map, p.v_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
+                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2))
+    return cudaErrorNotSupported;
+  cudaError_t e = cudaFuncSetAttribute(attention_mq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kTcSmemBytes);
+  if (e != cudaSuccess) return e;
+  const int rows_total = mp.n_q * p.group;
+  const int n_rb = (rows_total + kTcRows - 1) / kTcRows;
+  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(mp.n_chunks_grid) : 1u;
+  dim3 grid(chunks, p.geom.num_kv_heads * n_rb, p.batch);
+  attention_mq_tc_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(k_map, v_map, mp);
+  return cudaGetLastError();
+}
+
+}  // namespace pda

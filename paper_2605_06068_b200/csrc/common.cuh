@@ -109,6 +109,9 @@ cudaError_t launch_reduce(const float* part_o, const float* part_lse, const int3
                           int32_t first_chunks, int32_t tokens_per_seq, __nv_bfloat16* out,
                           cudaStream_t stream);
 bool attention_mq_supports(const MqParams& mp);
+// tcgen05 + TMEM version (bf16 KV, head_dim 128)
+bool attention_mq_tc_supports(const MqParams& mp);
+cudaError_t launch_attention_mq_tc(const MqParams& mp, cudaStream_t stream);
 cudaError_t launch_attention_mq(const MqParams& mp, cudaStream_t stream);
 cudaError_t launch_kv_append_tokens(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                     const CacheGeom& g, const int32_t* block_table, int32_t bt_stride,

@@ -9,7 +9,10 @@
 
 namespace pda {
 
-constexpr uint32_t kSpinLimit = 1u << 22;  // polls before a bounded mbarrier wait gives up
+// A bounded mbarrier wait polls try_wait at most kSpinLimit times, each poll suspended for at
+// most kSuspendNs: it gives up after roughly a second instead of hanging.
+constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kSuspendNs = 1000;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -24,9 +27,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
 }
 // Bounded wait: false if the phase did not complete within kSpinLimit polls.

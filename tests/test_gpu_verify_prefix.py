@@ -11,6 +11,9 @@ from util import DeviceWorkload, assert_close, bf16_tensor, bf16_to_bits, bf16_t
 
 pytestmark = pytest.mark.gpu
 
+# the multi-query kernels: tcgen05 + TMEM where it applies (bf16, head_dim 128), else / forced mma.sync
+MQ = [pytest.param(0, id="tcgen05"), pytest.param(pda.PDA_FLAG_MQ_MMA_SYNC, id="mma_sync")]
+
 
 def verify_inputs(w, T, seed):
     rng = np.random.default_rng(seed)
@@ -21,12 +24,13 @@ def verify_inputs(w, T, seed):
     return q, kn, vn
 
 
-@pytest.mark.parametrize("T", [1, 4, 16])
+@pytest.mark.parametrize("flags", MQ)
+@pytest.mark.parametrize("T", [1, 4, 16, 40])
 @pytest.mark.parametrize("shape", [(8, 2, 64), (32, 8, 128), (64, 8, 128), (8, 8, 128)],
                          ids=lambda s: f"Hq{s[0]}kv{s[1]}D{s[2]}")
-def test_verify_attention_and_block_append(oracle, shape, T):
+def test_verify_attention_and_block_append(oracle, shape, T, flags):
     Hq, Hkv, D = shape
-    lens = [16, 17, 31, 40, 100, 640, 1300]
+    lens = [40, 41, 63, 64, 100, 640, 1300]
     w = W.make_workload("verify", lens, Hq, Hkv, D, seed=19)
     q, kn, vn = verify_inputs(w, T, 20)
     k, v = w.k_cache.copy(), w.v_cache.copy()
@@ -39,7 +43,7 @@ def test_verify_attention_and_block_append(oracle, shape, T):
     assert (bf16_to_bits(dw.k_cache) == k).all() and (bf16_to_bits(dw.v_cache) == v).all()
     dq = bf16_tensor(q)
     out = pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
-                                     float(w.scale), status=dw.status)
+                                     float(w.scale), flags=flags, status=dw.status)
     assert_close(bf16_to_f64(out), ref, what=f"verify T={T} unsplit")
     for chunk in (64, 256):
         mc = pda.max_chunks(max(lens), chunk)
@@ -47,7 +51,7 @@ def test_verify_attention_and_block_append(oracle, shape, T):
         pl = torch.full((w.batch, T, Hq, mc), float("nan"), dtype=torch.float32, device="cuda")
         out_s = pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
                                            float(w.scale), chunk_tokens=chunk, part_o=po, part_lse=pl,
-                                           status=dw.status)
+                                           flags=flags, status=dw.status)
         assert_close(bf16_to_f64(out_s), ref, what=f"verify T={T} chunk {chunk}")
     # the last query token sees the whole sequence: same as plain decode attention (up to rounding)
     plain = pda.paged_decode_attention(dq[:, -1].contiguous(), dw.k_cache, dw.v_cache, dw.block_table,
@@ -85,9 +89,10 @@ def test_verify_attention_fp8_and_causal_needle(oracle):
     assert np.abs(out[0, :-1]).max() < 3.0    # N(0,1) averages, nowhere near 1..128
 
 
+@pytest.mark.parametrize("flags", MQ)
 @pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
 @pytest.mark.parametrize("B", [3, 40])
-def test_shared_prefix_cascade(oracle, kv_dtype, B):
+def test_shared_prefix_cascade(oracle, kv_dtype, B, flags):
     rng = np.random.default_rng(7)
     prefix = 512
     lens = prefix + rng.integers(0, 300, size=B)
@@ -106,7 +111,8 @@ def test_shared_prefix_cascade(oracle, kv_dtype, B):
         pl = torch.full((B, 32, mc), float("nan"), dtype=torch.float32, device="cuda")
         out = pda.paged_prefix_decode_attention(dw.q, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
                                                 float(w.scale), prefix, pchunk, chunk, po, pl,
-                                                k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+                                                k_scale=dw.k_scale, v_scale=dw.v_scale, flags=flags,
+                                                status=dw.status)
         assert_close(bf16_to_f64(out), ref, kv_dtype, what=f"cascade {kv_dtype} B={B} chunks {pchunk}/{chunk}")
     plain = dw.attend()
     assert np.abs(bf16_to_f64(plain) - bf16_to_f64(out)).max() < 2e-2
