@@ -5,24 +5,26 @@
 //
 // This is the part of the path that is a real dense contraction, so it runs as
 // UMMA tiles with accumulators in tensor memory:
-//   S[128 x 64]  = Q[128 x D] . K^T     per 4 pages: per page 8 tcgen05.mma of
-//                                        M128 x N16 x K16 (K-major A and B)
+//   S[128 x 64]  = Q[128 x D] . K^T     per 4 pages: 8 tcgen05.mma of M128 x N64 x K16
+//                                        (K-major A and B; the 4 pages' rows are stacked)
 //   O[128 x D]  += P[128 x 64] . V      per page 1 tcgen05.mma M128 x N128 x K16
 //                                        (A = P from shared memory, B = V MN-major)
-// The (page, head) tiles land through the same 5-D TMA map as everywhere else:
-// [128-byte line][16 slots][128 B] with the 128-byte swizzle is already the
-// canonical UMMA layout, K-major for K (rows = tokens, contraction over d) and
-// MN-major for V (contraction over the 16 tokens of the page), so no data is
-// rearranged in shared memory.
+// The (page, head) tiles land through the same 5-D TMA maps as everywhere else: rows of
+// 128-byte lines with the 128-byte swizzle are already the canonical UMMA layouts, K-major
+// for K (rows = tokens, contraction over d; copied line by line so that the 4 pages of an
+// iteration stack to [line][64 tokens][128 B]) and MN-major for V (contraction over the 16
+// tokens of a page), so no data is rearranged in shared memory. One elected thread issues
+// the MMAs; few, wide instructions matter (a tcgen05.mma costs ~40-100 ns to issue here).
 //
 // Warp roles (6 warps): 0-3 softmax (thread t <-> TMEM lane t <-> query row t),
-// 4 TMA producer, 5 MMA issue + TMEM allocation. Per iteration of 64 tokens:
-//   MMA warp:   wait stage -> S MMAs -> commit(bar_s) ; wait bar_p -> PV MMAs ->
-//               commit(stage empty), commit(bar_o)
-//   softmax:    wait bar_s -> tcgen05.ld S -> scale, mask, row max (thread-local)
-//               -> wait bar_o of the previous iteration -> (rarely) rescale O in
-//               TMEM when the running max grew by more than 2^8 -> P = exp2(..)
-//               as bf16 into the swizzled P tile -> arrive(bar_p)
+// 4 TMA producer, 5 MMA issue + TMEM allocation. S and P are double-buffered so that
+// the tensor core computes S of iteration i+1 while the softmax warps work on i:
+//   MMA warp:   S(0); then per iteration i: S(i+1) -> commit(bar_s[(i+1)&1]);
+//               wait bar_p[i&1] -> PV(i) -> commit(stage empty), commit(bar_pv[i&1])
+//   softmax:    wait bar_s[i&1] -> tcgen05.ld S -> scale, mask, row max (thread-local)
+//               -> wait bar_pv of iteration i-2 (its P buffer is free again) -> (rarely,
+//               after waiting for PV(i-1)) rescale O in TMEM when the running max grew by
+//               more than 2^8 -> P = exp2(..) as bf16 into the swizzled P tile -> arrive(bar_p[i&1])
 // All mbarrier waits are bounded; TMEM is always released before the CTA exits.
 #include "common.cuh"
 #include "tma_ptx.cuh"
@@ -36,13 +38,13 @@ constexpr int kTcRows = 128;            // query rows per CTA (UMMA M)
 constexpr int kTcPagesPerIter = 4;      // 64 tokens per iteration
 constexpr int kTcStages = 4;
 constexpr int kTcTileBytes = kPageSize * kTcD * 2;        // 4096: one K or V page tile
-constexpr int kTcPageBytes = 2 * kTcTileBytes;            // K then V
-constexpr int kTcStageBytes = kTcPagesPerIter * kTcPageBytes;  // 32 KB
+constexpr int kTcKBytes = kTcPagesPerIter * kTcTileBytes;  // 16 KB: K of 4 pages as [2 lines][64 tokens][128 B]
+constexpr int kTcStageBytes = 2 * kTcKBytes;               // 32 KB: K block, then 4 V page tiles
 constexpr int kTcQBytes = kTcRows * kTcD * 2;             // 32 KB: [2 lines][128 rows][128 B]
-constexpr int kTcPBytes = kTcRows * 128;                  // 16 KB: [128 rows][64 tokens] bf16
-constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcQBytes + kTcPBytes + 256 + 1024;
+constexpr int kTcPBytes = kTcRows * 128;                  // 16 KB: [128 rows][64 tokens] bf16 (two of them)
+constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcQBytes + 2 * kTcPBytes + 256 + 1024;
 constexpr int kTcThreads = 192;
-constexpr uint32_t kTmemCols = 256;     // S: columns 0..63, O: columns 64..191
+constexpr uint32_t kTmemCols = 256;     // S buffers: columns 0..63 and 64..127, O: columns 128..255
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the max grows this much
 
 __device__ __forceinline__ void mbar_arrive_tc(uint32_t bar) {
@@ -108,8 +110,8 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_smem = smem + kTcStages * kTcStageBytes;
   uint8_t* p_smem = q_smem + kTcQBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(p_smem + kTcPBytes);  // full[4], empty[4], s, p, o
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 3);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(p_smem + 2 * kTcPBytes);  // full[], empty[], s[2], p[2], pv[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 6);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -139,15 +141,17 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 
   const uint32_t ring = smem_u32(smem);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
-  const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 8, bar_o = bar_p + 8;
+  const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
     }
-    mbar_init(bar_s, 1);
-    mbar_init(bar_p, 4);   // one arrival per softmax warp
-    mbar_init(bar_o, 1);
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(bar_s + 8 * k, 1);
+      mbar_init(bar_p + 8 * k, 4);   // one arrival per softmax warp
+      mbar_init(bar_pv + 8 * k, 1);
+    }
     *cta_err = 0;
     fence_mbar_init();
     fence_proxy_async();
@@ -176,7 +180,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 64;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 128;  // S buffer k at tmem_s + 64 k
 
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
 
@@ -198,34 +202,41 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
       const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
-      if (lane == 0) mbar_expect_tx(full0 + 8 * s, n_here * kTcPageBytes);
+      if (lane == 0) mbar_expect_tx(full0 + 8 * s, n_here * 2 * kTcTileBytes);
       for (int j = 0; j < n_here; ++j) {
         const int page_raw = __shfl_sync(0xffffffffu, pg, (it & 7) * kTcPagesPerIter + j);
         if (page_raw < 0) bad = true;
         if (lane == 0) {
-          const uint32_t dst = ring + s * kTcStageBytes + j * kTcPageBytes;
-          tma_load_5d(dst, &k_map, full0 + 8 * s, 0, 0, 0, g, max(page_raw, 0));
-          tma_load_5d(dst + kTcTileBytes, &v_map, full0 + 8 * s, 0, 0, 0, g, max(page_raw, 0));
+          const uint32_t stage = ring + s * kTcStageBytes;
+          const int page = max(page_raw, 0);
+          // K: one copy per 128-byte line so that page j's 16 rows follow page j-1's in each line block
+          tma_load_5d(stage + j * (kPageSize * 128), &k_map, full0 + 8 * s, 0, 0, 0, g, page);
+          tma_load_5d(stage + kTcKBytes / 2 + j * (kPageSize * 128), &k_map, full0 + 8 * s, 0, 0, 1, g, page);
+          tma_load_5d(stage + kTcKBytes + j * kTcTileBytes, &v_map, full0 + 8 * s, 0, 0, 0, g, page);
         }
       }
     }
     if (bad && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
   } else if (warp == 5) {
     // ================= MMA issue =================
-    constexpr uint32_t idesc_s = tc_idesc(16, false);
+    constexpr uint32_t idesc_s = tc_idesc(kTcPagesPerIter * kPageSize, false);
     constexpr uint32_t idesc_pv = tc_idesc(D, true);
     const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
-    for (int it = 0; it < n_iters; ++it) {
+    uint64_t q_desc[D / 16];
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks)
+      q_desc[ks] = tc_desc(q_addr + (ks >> 2) * (kTcRows * 128) + (ks & 3) * 32, 16, 1024);
+    // Waits for stage `it`, clears the rows past the sequence end in V, issues S(it) = Q . K^T
+    auto issue_s = [&](int it) -> bool {
       const int s = it % kTcStages;
       bool ok = mbar_wait_bounded(full0 + 8 * s, (it / kTcStages) & 1);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
+      if (!ok) return false;
       const uint32_t stage = ring + s * kTcStageBytes;
       const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
-      // rows of the sequence's last page past its end may hold anything: clear them in V
       const int tail = L - (page0 + it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
       if (tail < kPageSize) {
-        const uint32_t vt = stage + (n_here - 1) * kTcPageBytes + kTcTileBytes;
+        const uint32_t vt = stage + kTcKBytes + (n_here - 1) * kTcTileBytes;
         for (int i = lane; i < (kPageSize - tail) * 16; i += 32) {
           const int r = tail + i / 16, ch = i % 16;
           asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_off(r, ch)), "r"(0));
@@ -235,36 +246,47 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       tc_fence_after();
       if (lane == 0) {
-        // S columns [16j, 16j+16) = Q . K_j^T, contraction over d in 8 steps of 16
-        for (int j = 0; j < n_here; ++j) {
-          const uint32_t kt = stage + j * kTcPageBytes;
+        const uint32_t d = tmem_s + 64 * (it & 1);
+        // S[:, 0..64) = Q . K^T over the 64 stacked token rows, contraction over d in 8 steps of 16
+        // (rows of pages that were not loaded hold stale data: those columns are masked later)
+        const uint64_t kd0 = tc_desc(stage, 16, 1024);
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const uint64_t a = tc_desc(q_addr + (ks >> 2) * (kTcRows * 128) + (ks & 3) * 32, 16, 1024);
-            const uint64_t bd = tc_desc(kt + (ks >> 2) * (kPageSize * 128) + (ks & 3) * 32, 16, 1024);
-            tc_mma(tmem_s + 16 * j, a, bd, idesc_s, ks > 0 ? 1u : 0u);
-          }
+        for (int ks = 0; ks < D / 16; ++ks) {
+          // descriptor start addresses are in 16-byte units: +2 per k-step, next line block further on
+          const uint64_t bd = kd0 + static_cast<uint64_t>((ks >> 2) * (kTcKBytes / 2 / 16) + (ks & 3) * 2);
+          tc_mma(d, q_desc[ks], bd, idesc_s, ks > 0 ? 1u : 0u);
         }
-        tc_commit(bar_s);
+        tc_commit(bar_s + 8 * (it & 1));
       }
       __syncwarp();
-      ok = mbar_wait_bounded(bar_p, it & 1);
+      return true;
+    };
+    bool ok = n_iters > 0 ? issue_s(0) : true;
+    for (int it = 0; it < n_iters && ok; ++it) {
+      // S(it+1) goes to the other S buffer, which softmax(it-1) has released (it arrived on bar_p
+      // before PV(it-1) was issued)
+      if (it + 1 < n_iters) ok = issue_s(it + 1);
+      if (!ok) break;
+      ok = mbar_wait_bounded(bar_p + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
+      if (!ok) break;
       tc_fence_after();
       if (lane == 0) {
+        const int s = it % kTcStages;
+        const uint32_t stage = ring + s * kTcStageBytes;
+        const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
         // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page, V read MN-major
-        for (int j = 0; j < n_here; ++j) {
-          const uint32_t vt = stage + j * kTcPageBytes + kTcTileBytes;
-          const uint64_t a = tc_desc(p_addr + j * 32, 16, 1024);
-          const uint64_t bd = tc_desc(vt, kPageSize * 128, 1024);  // LBO: next 64 columns of d, SBO: next 8 tokens
-          tc_mma(tmem_o, a, bd, idesc_pv, (it > 0 || j > 0) ? 1u : 0u);
-        }
-        tc_commit(empty0 + 8 * s);  // the stage may be refilled once these MMAs have read it
-        tc_commit(bar_o);
+        const uint64_t pd0 = tc_desc(p_addr + (it & 1) * kTcPBytes, 16, 1024);
+        const uint64_t vd0 = tc_desc(stage + kTcKBytes, kPageSize * 128, 1024);  // LBO: next 64 columns of d, SBO: next 8 tokens
+        for (int j = 0; j < n_here; ++j)
+          tc_mma(tmem_o, pd0 + static_cast<uint64_t>(2 * j), vd0 + static_cast<uint64_t>(j * (kTcTileBytes / 16)),
+                 idesc_pv, (it > 0 || j > 0) ? 1u : 0u);
+        tc_commit(empty0 + 8 * s);            // the stage may be refilled once these MMAs have read it
+        tc_commit(bar_pv + 8 * (it & 1));     // P buffer free again, O updated
       }
       __syncwarp();
     }
+    if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   } else {
     // ================= softmax: thread t owns query row t =================
     const int r = rb * kTcRows + tid;
@@ -276,13 +298,13 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     float l = 0.f;
     bool alive = true;
     for (int it = 0; it < n_iters && alive; ++it) {
-      bool ok = mbar_wait_bounded(bar_s, it & 1);
+      bool ok = mbar_wait_bounded(bar_s + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
       tc_fence_after();
       uint32_t sv[2][32];
-      tmem_ld32(tmem_s + lane_base, sv[0]);
-      tmem_ld32(tmem_s + lane_base + 32, sv[1]);
+      tmem_ld32(tmem_s + 64 * (it & 1) + lane_base, sv[0]);
+      tmem_ld32(tmem_s + 64 * (it & 1) + lane_base + 32, sv[1]);
       tmem_wait_ld();
       const int tok0 = (page0 + it * kTcPagesPerIter) * kPageSize;
       const int n_vis = min(lim, t1) - tok0;  // visible columns of this row in this iteration (may be <= 0)
@@ -300,12 +322,19 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       float m_new = m_ref;
       if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = fmaxf(m_ref, mx);
       const bool need = m_new != m_ref && m_ref != -INFINITY;
-      if (it > 0) {
-        ok = mbar_wait_bounded(bar_o, (it - 1) & 1);  // previous PV done: O is stable, P tile is free
+      if (it >= 2) {  // PV(it-2) has finished reading the P buffer this iteration writes
+        ok = mbar_wait_bounded(bar_pv + 8 * (it & 1), ((it >> 1) - 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
-        tc_fence_after();
+      }
+      if (it > 0) {
         if (__any_sync(0xffffffffu, need)) {
+          // O may only be touched once PV(it-1) has completed (PV(it) is not issued before this
+          // warp arrives on bar_p below)
+          ok = mbar_wait_bounded(bar_pv + 8 * ((it - 1) & 1), ((it - 1) >> 1) & 1);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
+          tc_fence_after();
           const float alpha = need ? ex2(m_ref - m_new) : 1.f;
           l *= alpha;
 #pragma unroll
@@ -324,7 +353,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       const float ref = m_ref == -INFINITY ? 0.f : m_ref;
       // P = exp2(S - ref) as bf16 into row `tid` of the swizzled [128 rows][128 B] tile
       float lsum = 0.f;
-      const uint32_t prow = smem_u32(p_smem) + tid * 128;
+      const uint32_t prow = smem_u32(p_smem) + (it & 1) * kTcPBytes + tid * 128;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
         uint32_t w[4];
@@ -343,13 +372,13 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       fence_proxy_async();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_tc(bar_p);
+      if (lane == 0) mbar_arrive_tc(bar_p + 8 * (it & 1));
     }
 
     // ---- finalise this row
     bool ok = true;
     if (alive && n_iters > 0) {
-      ok = mbar_wait_bounded(bar_o, (n_iters - 1) & 1);
+      ok = mbar_wait_bounded(bar_pv + 8 * ((n_iters - 1) & 1), ((n_iters - 1) >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
       tc_fence_after();
@@ -421,7 +450,7 @@ cudaError_t launch_attention_mq_tc(const MqParams& mp, cudaStream_t stream) {
   const AttnParams& p = mp.a;
   alignas(64) CUtensorMap k_map, v_map;
   if (!make_cache_tensor_map(&k_map, p.k_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
-                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2) ||
+                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2, /*box_lines=*/1) ||
       !make_cache_tensor_map(&v_map, p.v_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
                              p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2))
     return cudaErrorNotSupported;

@@ -510,7 +510,7 @@ EncodeFn encode_fn() {
 
 bool make_cache_tensor_map(CUtensorMap* map, const void* base, int64_t page_stride,
                            int64_t head_stride, int64_t slot_stride, int num_pages,
-                           int num_kv_heads, int head_dim, int eb) {
+                           int num_kv_heads, int head_dim, int eb, int box_lines) {
   EncodeFn enc = encode_fn();
   if (!enc) return false;
   const cuuint64_t line_elems = 128 / eb;
@@ -520,7 +520,8 @@ bool make_cache_tensor_map(CUtensorMap* map, const void* base, int64_t page_stri
   cuuint64_t strides[4] = {static_cast<cuuint64_t>(slot_stride) * eb, 128,
                            static_cast<cuuint64_t>(head_stride) * eb,
                            static_cast<cuuint64_t>(page_stride) * eb};
-  cuuint32_t box[5] = {static_cast<cuuint32_t>(line_elems), kPageSize, static_cast<cuuint32_t>(lines), 1, 1};
+  cuuint32_t box[5] = {static_cast<cuuint32_t>(line_elems), kPageSize,
+                       static_cast<cuuint32_t>(box_lines > 0 ? box_lines : lines), 1, 1};
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   const CUresult r = enc(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 5,
                          const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,

@@ -107,9 +107,10 @@ __device__ __forceinline__ uint32_t tile_off(int r, int chunk) {
 }
 
 // Host: 5-D tiled tensor map of a KV cache, dims (byte lane within a 128-byte
-// line, slot, line of the row, head, page), box = one (page, head) tile.
+// line, slot, line of the row, head, page), box = one (page, head) tile, or only
+// `box_lines` of its 128-byte lines when box_lines > 0.
 bool make_cache_tensor_map(CUtensorMap* map, const void* base, int64_t page_stride,
                            int64_t head_stride, int64_t slot_stride, int num_pages,
-                           int num_kv_heads, int head_dim, int elem_bytes);
+                           int num_kv_heads, int head_dim, int elem_bytes, int box_lines = 0);
 
 }  // namespace pda
