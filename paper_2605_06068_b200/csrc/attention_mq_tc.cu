@@ -118,8 +118,24 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const int G = p.group, T = mp.n_q;
   const int rows_total = T * G;
   const int n_rb = (rows_total + kTcRows - 1) / kTcRows;
-  const int c = blockIdx.x, g = blockIdx.y / n_rb, rb = blockIdx.y % n_rb, b = blockIdx.z;
+  const int c = blockIdx.x, g = blockIdx.y / n_rb, rb = blockIdx.y % n_rb;
   const bool split = p.chunk_tokens > 0;
+  int b = blockIdx.z;
+  if (!split && mp.kv_len_fixed == 0 && p.batch > 1 && p.batch <= 128) {  // (ranking costs O(batch^2/threads))
+    // unsplit units differ in length: the CTA with blockIdx.z = r serves the r-th longest sequence
+    int* lens = reinterpret_cast<int*>(smem);
+    for (int j = tid; j < p.batch; j += kTcThreads) lens[j] = max(p.seq_lens[j], 0);
+    __syncthreads();
+    for (int j = tid; j < p.batch; j += kTcThreads) {
+      const int Lj = lens[j];
+      int rank = 0;
+      for (int i = 0; i < p.batch; ++i) rank += (lens[i] > Lj) || (lens[i] == Lj && i < j);
+      if (rank == static_cast<int>(blockIdx.z)) *cta_err = j;
+    }
+    __syncthreads();
+    b = *cta_err;
+    __syncthreads();  // lens aliases the ring and cta_err is reused below
+  }
 
   const int L = mp.kv_len_fixed > 0 ? mp.kv_len_fixed : max(p.seq_lens[b], 0);
   int t0 = p.first_token, t1 = L;
