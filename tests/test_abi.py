@@ -94,3 +94,42 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(pda, "LIB_PATH", "/nonexistent/libpda.so")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         pda.lib()
+
+
+def test_new_entry_points_validate_without_a_gpu(lib):
+    d = desc()
+    P = 0x1000
+    # paged_decode_step: k_new without v_new, missing out, e4m3 cache with an append
+    step = lambda **kw: lib.paged_decode_step(
+        kw.get("q", P), kw.get("kn", P), kw.get("vn", P), P, P, C.byref(kw.get("d", d)), None, None, P, 4, P,
+        kw.get("batch", 1), 32, 0.1, kw.get("chunk", 0), kw.get("out", P), None, None, 0, None, None, None)
+    assert step(vn=None) == -1
+    assert step(out=None) == -1
+    assert step(batch=0) == 0
+    assert step(chunk=8) == -1
+    # window must be non-negative
+    assert lib.paged_window_decode_attention(P, P, P, C.byref(d), None, None, P, 4, P, 1, 32, 0.1, -1, 0,
+                                             P, None, None, 0, 0, None, None) == -1
+    # verify: token count, batch * tokens limit
+    ver = lambda T, batch=1: lib.paged_verify_attention(P, P, P, C.byref(d), None, None, P, 4, P, batch, 32, T,
+                                                        0.1, 0, P, None, None, 0, 0, None, None)
+    assert ver(0) == -1 and ver(5000) == -1 and ver(16, batch=5000) == -4 and ver(16, batch=0) == 0
+    # shared prefix: prefix must be page-aligned, chunks positive, max_chunks must leave room for suffixes
+    pre = lambda prefix, pchunk, chunk, mc: lib.paged_prefix_decode_attention(
+        P, P, P, C.byref(d), None, None, P, 64, P, 2, 32, 0.1, prefix, pchunk, chunk, P, P, P, mc, 0, None, None)
+    assert pre(100, 64, 64, 8) == -1
+    assert pre(128, 0, 64, 8) == -1
+    assert pre(128, 64, 0, 8) == -1
+    assert pre(128, 64, 64, 2) == -1
+    assert pre(4096, 64, 64, 100) == -1       # prefix longer than the block table can hold
+    # fp8 append needs an e4m3 cache and both scale arrays
+    assert lib.kv_append_fp8(P, P, P, P, C.byref(d), P, P, P, 4, P, 1, None, None) == -2
+    d8 = desc(dtype=1, page_stride=8 * 16 * 128, head_stride=16 * 128)
+    assert lib.kv_append_fp8(P, P, P, P, C.byref(d8), None, P, P, 4, P, 1, None, None) == -1
+    assert lib.kv_append_tokens(P, P, P, P, C.byref(d), P, 4, P, 1, -1, None, None) == -1
+    assert lib.kv_append_tokens(P, P, P, P, C.byref(d), P, 4, P, 1, 0, None, None) == 0
+    assert lib.pda_workspace_ints(64, 8) == 514 and lib.pda_workspace_ints(-1, 8) == -1
+    assert lib.pda_advance_seq_lens(None, 4, 1, None) == -1 and lib.pda_advance_seq_lens(None, 0, 1, None) == 0
+    # the allocation-free entry point rejects oversize problems before touching the device
+    assert lib.paged_decode_attention_static(P, P, P, C.byref(d), None, None, P, 4, P, 64, 32, 0.1, 16,
+                                             4096, P, None, None) == -4
