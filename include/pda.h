@@ -251,6 +251,13 @@ int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_
                         int32_t chunk_tokens, int32_t max_chunks, void* out,
                         pda_stream_t stream);
 
+/* Tuning knob (process-wide, host side): an unsplit paged_decode_step with a workspace
+ * and batch <= 256 runs on the persistent kernel (resident CTAs looping over (sequence, kv
+ * head) units through the workspace's work ticket, longest first) once there are at least
+ * min_units_per_cta units per resident CTA (2 per SM); below that, one CTA per unit is
+ * faster. Default 6. 0 always selects the persistent kernel where it applies (tests). */
+int pda_set_persistent_threshold(int32_t min_units_per_cta);
+
 /* Number of int32 the `workspace` of paged_decode_step needs: 2 + batch*num_kv_heads. */
 int pda_workspace_ints(int32_t batch, int32_t num_kv_heads);
 
@@ -265,8 +272,8 @@ int pda_workspace_ints(int32_t batch, int32_t num_kv_heads);
  *              caller ONCE (e.g. at allocation); every call leaves it zeroed again,
  *              so consecutive calls on one stream may share it. Calls that can
  *              overlap on the GPU need separate workspaces. It carries the work
- *              per-(sequence, kv head) chunk counters (two leading ints are
- *              reserved). May be NULL when chunk_tokens == 0. After a
+ *              the work ticket of the persistent kernel (two leading ints)
+ *              and the per-(sequence, kv head) chunk counters. May be NULL when chunk_tokens == 0. After a
  *              PDA_DEV_TIMEOUT status, zero it again.
  * If chunk_tokens > 0 and workspace is NULL, or the shape is outside the fused
  * kernel's set (group size > 8, head_dim not 64/128), the step is

@@ -24,7 +24,8 @@ EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
            "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
            "paged_decode_step", "pda_advance_seq_lens", "paged_window_decode_attention", "kv_append_tokens",
-           "paged_verify_attention", "paged_prefix_decode_attention", "kv_append_fp8"]
+           "paged_verify_attention", "paged_prefix_decode_attention", "kv_append_fp8",
+           "pda_set_persistent_threshold"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
@@ -58,6 +59,7 @@ def lib():
         L.paged_decode_step_host.argtypes = [vp] * 5 + [vp] * 5 + [vp, vp, dp, i32, i32, i32, f32,
                                                                  i32, vp, vp, i32, vp, vp, vp, vp, vp]
         L.pda_workspace_ints.argtypes = [i32, i32]
+        L.pda_set_persistent_threshold.argtypes = [i32]
         L.kv_append_fp8.argtypes = [vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, vp, vp]
         L.kv_append_tokens.argtypes = [vp, vp, vp, vp, dp, vp, i32, vp, i32, i32, vp, vp]
         L.paged_verify_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, i32, f32,
@@ -322,3 +324,8 @@ def kv_append_fp8(k_new, v_new, k_cache, v_cache, k_scale, v_scale, block_table,
                              _ptr(k_scale), _ptr(v_scale), _ptr(block_table), block_table.stride(0),
                              _ptr(seq_lens), seq_lens.shape[0], _ptr(status), _stream(stream))
     _check(rc, "kv_append_fp8")
+
+
+def set_persistent_threshold(min_units_per_cta: int):
+    """Units per resident CTA from which the unsplit fused step uses the persistent kernel (0: always)."""
+    _check(lib().pda_set_persistent_threshold(int(min_units_per_cta)), "pda_set_persistent_threshold")

@@ -1,4 +1,5 @@
 // C ABI of libpda: argument validation on the host, then kernel dispatch.
+#include <atomic>
 #include <cstdint>
 
 #include "common.cuh"
@@ -7,6 +8,9 @@ namespace {
 
 using pda::AttnParams;
 using pda::CacheGeom;
+
+// units per resident CTA from which paged_decode_step uses the persistent kernel (unsplit launches)
+std::atomic<int> g_persist_min_units{6};
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -301,6 +305,12 @@ int paged_prefix_decode_attention(const void* q, const void* k_cache, const void
                                              static_cast<__nv_bfloat16*>(out), s));
 }
 
+int pda_set_persistent_threshold(int32_t min_units_per_cta) {
+  if (min_units_per_cta < 0) return PDA_ERR_INVALID_ARG;
+  g_persist_min_units.store(min_units_per_cta);
+  return PDA_OK;
+}
+
 int pda_workspace_ints(int32_t batch, int32_t num_kv_heads) {
   if (batch < 0 || num_kv_heads <= 0) return PDA_ERR_INVALID_ARG;
   const int64_t n = 2 + static_cast<int64_t>(batch) * num_kv_heads;
@@ -330,6 +340,8 @@ int paged_decode_step(const void* q, const void* k_new, const void* v_new, void*
   const bool can_fuse = pda::attention_tma_supports(p) && (chunk_tokens == 0 || workspace);
   if (can_fuse) {
     pda::StepParams sp{p, k_new, v_new, k_cache, v_cache, workspace, 1};
+    if (pda::attention_persist_supports(sp) && pda::attention_persist_preferred(sp, g_persist_min_units))
+      return static_cast<int>(pda::launch_attention_persist(sp, static_cast<cudaStream_t>(stream)));
     return static_cast<int>(pda::launch_step_tma(sp, static_cast<cudaStream_t>(stream)));
   }
   // shapes outside the fused kernel: the same step as separate launches

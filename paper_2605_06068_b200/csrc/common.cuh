@@ -102,6 +102,10 @@ cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream);
 bool attention_tma_supports(const AttnParams& p);
 // Fused step on the same kernel: optional append, optional in-kernel reduce (sp.fuse_reduce).
 cudaError_t launch_step_tma(const StepParams& sp, cudaStream_t stream);
+// Persistent form of the fused step for unsplit launches (needs the workspace's work ticket).
+bool attention_persist_supports(const StepParams& sp);
+bool attention_persist_preferred(const StepParams& sp, int min_units_per_cta);
+cudaError_t launch_attention_persist(const StepParams& sp, cudaStream_t stream);
 // Rows are (sequence, query token, head): tokens_per_seq query tokens share one seq_lens entry.
 cudaError_t launch_reduce(const float* part_o, const float* part_lse, const int32_t* seq_lens,
                           int32_t batch, int32_t num_q_heads, int32_t head_dim,

@@ -14,9 +14,18 @@ from util import assert_close, bf16_tensor, bf16_to_bits, bf16_to_f64
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["persistent", "per_unit"])
+def step_kernel(request):
+    pda.set_persistent_threshold(0 if request.param == "persistent" else 1 << 30)
+    yield request.param
+    pda.set_persistent_threshold(6)
+
+
 @pytest.mark.parametrize("chunk", [0, 32])
 @pytest.mark.parametrize("shape", [(8, 2, 64), (32, 8, 128)])
-def test_graph_replayed_decode_loop(oracle, chunk, shape):
+def test_graph_replayed_decode_loop(oracle, chunk, shape, step_kernel):
+    if chunk and step_kernel == "persistent":
+        pytest.skip("the persistent kernel serves unsplit launches only")
     Hq, Hkv, D = shape
     T = 20
     start = np.array([1, 14, 15, 16, 30, 47, 200], np.int32)
