@@ -19,6 +19,13 @@
 // are converted to f16 in registers (cvt.rn.f16x2.e4m3x2, exact); their
 // per-(page, head) scales multiply the scores (K) and the probabilities (V).
 //
+// The tile math lives in decode_tile.cuh. The same kernel is the fused decode step
+// (paged_decode_step): the warp that owns the sequence's last page patches the new token's
+// K/V rows into the landed tile and stores them to the cache (append); split units publish
+// their partial and the unit's last-arriving chunk (atomic count in the caller's workspace)
+// merges them all; unsplit launches serve the longest sequences first. A token range
+// (first_token, window) restricts the attended tokens; pages wholly outside it are not read.
+//
 // Every wait on an mbarrier is bounded; on expiry the CTA reports
 // PDA_DEV_TIMEOUT, waits (bounded) for its copies in flight and zero-fills its
 // output. TMA copies never use multicast.
@@ -29,7 +36,6 @@
 namespace pda {
 
 namespace {
-
 
 // ---- kernel ------------------------------------------------------------------------------
 
