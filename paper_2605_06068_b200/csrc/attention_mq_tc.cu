@@ -4,27 +4,33 @@
 // query rows (query tokens x group size) per CTA against one sequence's pages.
 //
 // This is the part of the path that is a real dense contraction, so it runs as
-// UMMA tiles with accumulators in tensor memory:
+// UMMA tiles with operands and accumulators in tensor memory (TMEM, 128 lanes = query rows):
 //   S[128 x 64]  = Q[128 x D] . K^T     per 4 pages: 8 tcgen05.mma of M128 x N64 x K16
-//                                        (K-major A and B; the 4 pages' rows are stacked)
+//                                        (A = Q in TMEM, B = K, K-major; the 4 pages' rows are stacked)
 //   O[128 x D]  += P[128 x 64] . V      per page 1 tcgen05.mma M128 x N128 x K16
-//                                        (A = P from shared memory, B = V MN-major)
-// The (page, head) tiles land through the same 5-D TMA maps as everywhere else: rows of
-// 128-byte lines with the 128-byte swizzle are already the canonical UMMA layouts, K-major
-// for K (rows = tokens, contraction over d; copied line by line so that the 4 pages of an
-// iteration stack to [line][64 tokens][128 B]) and MN-major for V (contraction over the 16
-// tokens of a page), so no data is rearranged in shared memory. One elected thread issues
-// the MMAs; few, wide instructions matter (a tcgen05.mma costs ~40-100 ns to issue here).
+//                                        (A = P in TMEM, B = V, MN-major)
+//   l[128]      += P[128 x 64] . 1      per page 1 tcgen05.mma M128 x N16 x K16 against a tile of ones:
+//                                        the row sums of exactly the bf16 P that multiplies V
+// Only K and V are read from shared memory by the tensor core (with A there too an N = 64 MMA is bound
+// by shared-memory bandwidth: 50 instead of 33 clocks, measured). The (page, head) tiles land through
+// the same 5-D TMA maps as everywhere else: rows of 128-byte lines with the 128-byte swizzle are already
+// the canonical UMMA layouts, K-major for K (rows = tokens, contraction over d; copied line by line so
+// that the 4 pages of an iteration stack to [line][64 tokens][128 B]) and MN-major for V (contraction
+// over the 16 tokens of a page), so no data is rearranged in shared memory.
 //
-// Warp roles (6 warps): 0-3 softmax (thread t <-> TMEM lane t <-> query row t),
-// 4 TMA producer, 5 MMA issue + TMEM allocation. S and P are double-buffered so that
-// the tensor core computes S of iteration i+1 while the softmax warps work on i:
+// Warp roles (6 warps): 0-3 softmax (thread t <-> TMEM lane t <-> query row t), 4 TMA producer,
+// 5 MMA issue + TMEM allocation. The producer and MMA warps stay converged and issue through one
+// elected lane with predicated instructions and warp-uniform operands: issued from inside a divergent
+// branch, a TMA copy or an MMA cost 90-200 clocks each here and the issuing thread was the bottleneck;
+// this way they cost 25-35. S and P are double-buffered so that the tensor core computes S of
+// iteration i+1 while the softmax warps work on i:
 //   MMA warp:   S(0); then per iteration i: S(i+1) -> commit(bar_s[(i+1)&1]);
-//               wait bar_p[i&1] -> PV(i) -> commit(stage empty), commit(bar_pv[i&1])
-//   softmax:    wait bar_s[i&1] -> tcgen05.ld S -> scale, mask, row max (thread-local)
-//               -> wait bar_pv of iteration i-2 (its P buffer is free again) -> (rarely,
-//               after waiting for PV(i-1)) rescale O in TMEM when the running max grew by
-//               more than 2^8 -> P = exp2(..) as bf16 into the swizzled P tile -> arrive(bar_p[i&1])
+//               wait bar_p[i&1] -> PV(i), l(i) -> commit(stage empty), commit(bar_pv[i&1])
+//   softmax:    wait bar_s[i&1] -> tcgen05.ld S -> mask (boundary tiles), row max of the raw scores
+//               -> (rarely, after waiting for PV(i-1)) rescale O and l in TMEM when the running max
+//               grew by more than 2^8 -> P = exp2(S * scale - ref) as bf16 pairs (packed f32x2 FMA,
+//               one exp2 per element: the 16/clock/SM exp2 unit bounds these warps) -> tcgen05.st P
+//               -> arrive(bar_p[i&1])
 // All mbarrier waits are bounded; TMEM is always released before the CTA exits.
 #include "common.cuh"
 #include "tma_ptx.cuh"
@@ -36,32 +42,66 @@ namespace {
 constexpr int kTcD = 128;               // head_dim
 constexpr int kTcRows = 128;            // query rows per CTA (UMMA M)
 constexpr int kTcPagesPerIter = 4;      // 64 tokens per iteration
-constexpr int kTcStages = 4;
+constexpr int kTcStages = 5;
 constexpr int kTcTileBytes = kPageSize * kTcD * 2;        // 4096: one K or V page tile
 constexpr int kTcKBytes = kTcPagesPerIter * kTcTileBytes;  // 16 KB: K of 4 pages as [2 lines][64 tokens][128 B]
 constexpr int kTcStageBytes = 2 * kTcKBytes;               // 32 KB: K block, then 4 V page tiles
-constexpr int kTcQBytes = kTcRows * kTcD * 2;             // 32 KB: [2 lines][128 rows][128 B]
-constexpr int kTcPBytes = kTcRows * 128;                  // 16 KB: [128 rows][64 tokens] bf16 (two of them)
-constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcQBytes + 2 * kTcPBytes + 256 + 1024;
+constexpr int kTcOnesBytes = 2048;                         // bf16 ones: B operand [16 tokens][16 columns] of the row-sum MMA
+constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcOnesBytes + 256 + 1024;
 constexpr int kTcThreads = 192;
-constexpr uint32_t kTmemCols = 256;     // S buffers: columns 0..63 and 64..127, O: columns 128..255
+// Tensor memory columns (32-bit each, 128 lanes = query rows): S buffers 0..63 and 64..127 (f32),
+// O 128..255 (f32), Q 256..319 (bf16 pairs along d), P buffers 320..351 and 352..383 (bf16 pairs
+// along tokens). Allocations are powers of two.
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemO = 128, kTmemQ = 256, kTmemP = 320, kTmemL = 384;  // l: row sums of P, 16 columns (all equal)
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the max grows this much
 
+// Spinning bounded wait (no suspension): the waits on the MMA/softmax hand-off are short and on the
+// critical path, where the wake-up latency of a suspended try_wait shows.
+__device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < (1u << 24); ++i)
+    if (mbar_test_wait(bar, parity)) return true;
+  return false;
+}
 __device__ __forceinline__ void mbar_arrive_tc(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// The MMA warp stays converged: one elected lane (the same one every time) issues, the instruction is
+// predicated rather than branched around, so warp-uniform operands can stay in uniform registers.
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t is_leader;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(is_leader));
+  return is_leader;
 }
-// D[tmem] (+)= A[smem desc] . B[smem desc]; accumulate == 0 overwrites D
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] . B[smem descriptor]; accumulate == 0 overwrites D. A is read from tensor memory
+// (lane = row, 32-bit column = two consecutive k elements).
+__device__ __forceinline__ void tc_mma_ts_if(uint32_t leader, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                             uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+      "{\n\t.reg .pred pe, pa;\n\tsetp.ne.b32 pe, %5, 0;\n\tsetp.ne.b32 pa, %4, 0;\n\t"
+      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pa;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void tc_commit_if(uint32_t leader, uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %1, 0;\n\t"
+      "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_if(uint32_t leader, uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                               int c2, int c3, int c4) {
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %6, 0;\n\t"
+      "@pe cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {0, 0, %3, %4, %5}], [%2];\n\t}"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c2), "r"(c3), "r"(c4), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_if(uint32_t leader, uint32_t bar, uint32_t bytes) {
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %2, 0;\n\t"
+      "@pe mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(bar), "r"(bytes), "r"(leader) : "memory");
 }
 // Shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field.
 __device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -98,6 +138,20 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+// Packed pairs of f32 (sm_100): one instruction per two elements in the softmax inner loops.
+__device__ __forceinline__ uint64_t f32x2(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void f32x2_split(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -108,9 +162,8 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   constexpr int D = kTcD;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* q_smem = smem + kTcStages * kTcStageBytes;
-  uint8_t* p_smem = q_smem + kTcQBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(p_smem + 2 * kTcPBytes);  // full[], empty[], s[2], p[2], pv[2]
+  uint8_t* ones_smem = smem + kTcStages * kTcStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes);  // full[], empty[], s[2], p[2], pv[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 6);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
 
@@ -158,6 +211,8 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t ring = smem_u32(smem);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
+  for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads) reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;
+  fence_proxy_async();  // read by the tensor core through the async proxy
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full0 + 8 * s, 1);
@@ -178,37 +233,49 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
 
-  // ---- Q tile: row r -> (query token r / G, head r % G), written in the swizzled K-major layout
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTmemO;  // S buffer k at tmem_s + 64 k
+  const uint32_t tmem_q = tmem_base + kTmemQ, tmem_p = tmem_base + kTmemP;  // P buffer k at tmem_p + 32 k
+
+  // ---- Q: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of S = Q . K^T
   if (warp < 4) {
     const int r = rb * kTcRows + tid;
     const bool valid = r < rows_total;
     const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
     const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
 #pragma unroll
-    for (int ch = 0; ch < 16; ++ch) {
-      const uint4 v = valid ? src[ch] : make_uint4(0u, 0u, 0u, 0u);
-      const uint32_t dst = smem_u32(q_smem) + (ch >> 3) * (kTcRows * 128) + tid * 128 + (((ch & 7) ^ (tid & 7)) << 4);
-      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+    for (int h = 0; h < 2; ++h) {
+      uint32_t qv[32];
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        const uint4 v = valid ? src[h * 8 + ch] : make_uint4(0u, 0u, 0u, 0u);
+        qv[4 * ch] = v.x; qv[4 * ch + 1] = v.y; qv[4 * ch + 2] = v.z; qv[4 * ch + 3] = v.w;
+      }
+      tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32 * h, qv);
     }
-    fence_proxy_async();  // the tensor core reads this tile through the async proxy
+    tmem_wait_st();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 128;  // S buffer k at tmem_s + 64 k
 
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
 
   if (warp == 4) {
     // ================= TMA producer =================
+    const uint32_t leader = elect_one();
+    const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
+    const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     bool bad = false;
     int pg = 0;
-    for (int it = 0; it < n_iters; ++it) {
+    for (int it = 0; it < u_iters; ++it) {
       const int s = it % kTcStages;
       if ((it & 7) == 0) {  // page ids of the next 8 iterations (32 pages), one per lane
         pg = 0;
-        if (it * kTcPagesPerIter + lane < n_pages) {
+        if (it * kTcPagesPerIter + lane < u_pages) {
           const int v = table[page0 + it * kTcPagesPerIter + lane];
           pg = (v < 0 || v >= p.geom.num_pages) ? -1 : v;
         }
@@ -217,19 +284,23 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       if (it >= kTcStages) ok = mbar_wait_bounded(empty0 + 8 * s, ((it / kTcStages) - 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
-      const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
-      if (lane == 0) mbar_expect_tx(full0 + 8 * s, n_here * 2 * kTcTileBytes);
-      for (int j = 0; j < n_here; ++j) {
+      const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
+      const uint32_t stage = ring + s * kTcStageBytes, bar = full0 + 8 * s;
+      mbar_expect_tx_if(leader, bar, n_here * 2 * kTcTileBytes);
+      // K: one copy per 128-byte line so that page j's 16 rows follow page j-1's in each line block
+      auto load_page = [&](int j) {
         const int page_raw = __shfl_sync(0xffffffffu, pg, (it & 7) * kTcPagesPerIter + j);
-        if (page_raw < 0) bad = true;
-        if (lane == 0) {
-          const uint32_t stage = ring + s * kTcStageBytes;
-          const int page = max(page_raw, 0);
-          // K: one copy per 128-byte line so that page j's 16 rows follow page j-1's in each line block
-          tma_load_5d(stage + j * (kPageSize * 128), &k_map, full0 + 8 * s, 0, 0, 0, g, page);
-          tma_load_5d(stage + kTcKBytes / 2 + j * (kPageSize * 128), &k_map, full0 + 8 * s, 0, 0, 1, g, page);
-          tma_load_5d(stage + kTcKBytes + j * kTcTileBytes, &v_map, full0 + 8 * s, 0, 0, 0, g, page);
-        }
+        bad |= page_raw < 0;
+        const int page = max(page_raw, 0);
+        tma_load_5d_if(leader, stage + j * (kPageSize * 128), &k_map, bar, 0, g, page);
+        tma_load_5d_if(leader, stage + kTcKBytes / 2 + j * (kPageSize * 128), &k_map, bar, 1, g, page);
+        tma_load_5d_if(leader, stage + kTcKBytes + j * kTcTileBytes, &v_map, bar, 0, g, page);
+      };
+      if (n_here == kTcPagesPerIter) {
+#pragma unroll
+        for (int j = 0; j < kTcPagesPerIter; ++j) load_page(j);
+      } else {
+        for (int j = 0; j < n_here; ++j) load_page(j);
       }
     }
     if (bad && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
@@ -237,11 +308,14 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     // ================= MMA issue =================
     constexpr uint32_t idesc_s = tc_idesc(kTcPagesPerIter * kPageSize, false);
     constexpr uint32_t idesc_pv = tc_idesc(D, true);
-    const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
-    uint64_t q_desc[D / 16];
-#pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks)
-      q_desc[ks] = tc_desc(q_addr + (ks >> 2) * (kTcRows * 128) + (ks & 3) * 32, 16, 1024);
+    constexpr uint32_t idesc_l = tc_idesc(16, false);
+    const uint64_t ones_desc = tc_desc(smem_u32(ones_smem), 16, 1024);
+    const uint32_t leader = elect_one();
+    // warp-uniform copies (a shuffle from lane 0 tells the compiler so)
+    const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
+    const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
+    const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
+    const int u_tail0 = __shfl_sync(0xffffffffu, L - page0 * kPageSize, 0);  // tokens from the first page to the end
     // Waits for stage `it`, clears the rows past the sequence end in V, issues S(it) = Q . K^T
     auto issue_s = [&](int it) -> bool {
       const int s = it % kTcStages;
@@ -249,8 +323,8 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return false;
       const uint32_t stage = ring + s * kTcStageBytes;
-      const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
-      const int tail = L - (page0 + it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
+      const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
+      const int tail = u_tail0 - (it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
       if (tail < kPageSize) {
         const uint32_t vt = stage + kTcKBytes + (n_here - 1) * kTcTileBytes;
         for (int i = lane; i < (kPageSize - tail) * 16; i += 32) {
@@ -261,46 +335,49 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         __syncwarp();
       }
       tc_fence_after();
-      if (lane == 0) {
-        const uint32_t d = tmem_s + 64 * (it & 1);
-        // S[:, 0..64) = Q . K^T over the 64 stacked token rows, contraction over d in 8 steps of 16
-        // (rows of pages that were not loaded hold stale data: those columns are masked later)
-        const uint64_t kd0 = tc_desc(stage, 16, 1024);
+      const uint32_t d = u_tmem + 64 * (it & 1);
+      // S[:, 0..64) = Q . K^T over the 64 stacked token rows, contraction over d in 8 steps of 16
+      // (rows of pages that were not loaded hold stale data: those columns are masked later)
+      const uint64_t kd0 = tc_desc(stage, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          // descriptor start addresses are in 16-byte units: +2 per k-step, next line block further on
-          const uint64_t bd = kd0 + static_cast<uint64_t>((ks >> 2) * (kTcKBytes / 2 / 16) + (ks & 3) * 2);
-          tc_mma(d, q_desc[ks], bd, idesc_s, ks > 0 ? 1u : 0u);
-        }
-        tc_commit(bar_s + 8 * (it & 1));
+      for (int ks = 0; ks < D / 16; ++ks) {
+        // descriptor start addresses are in 16-byte units: +2 per k-step, next line block further on
+        const uint64_t bd = kd0 + static_cast<uint64_t>((ks >> 2) * (kTcKBytes / 2 / 16) + (ks & 3) * 2);
+        tc_mma_ts_if(leader, d, u_tmem + kTmemQ + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
       }
-      __syncwarp();
+      tc_commit_if(leader, bar_s + 8 * (it & 1));
       return true;
     };
-    bool ok = n_iters > 0 ? issue_s(0) : true;
-    for (int it = 0; it < n_iters && ok; ++it) {
+    bool ok = u_iters > 0 ? issue_s(0) : true;
+    for (int it = 0; it < u_iters && ok; ++it) {
       // S(it+1) goes to the other S buffer, which softmax(it-1) has released (it arrived on bar_p
       // before PV(it-1) was issued)
-      if (it + 1 < n_iters) ok = issue_s(it + 1);
+      if (it + 1 < u_iters) ok = issue_s(it + 1);
       if (!ok) break;
       ok = mbar_wait_bounded(bar_p + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      if (lane == 0) {
-        const int s = it % kTcStages;
-        const uint32_t stage = ring + s * kTcStageBytes;
-        const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
-        // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page, V read MN-major
-        const uint64_t pd0 = tc_desc(p_addr + (it & 1) * kTcPBytes, 16, 1024);
-        const uint64_t vd0 = tc_desc(stage + kTcKBytes, kPageSize * 128, 1024);  // LBO: next 64 columns of d, SBO: next 8 tokens
-        for (int j = 0; j < n_here; ++j)
-          tc_mma(tmem_o, pd0 + static_cast<uint64_t>(2 * j), vd0 + static_cast<uint64_t>(j * (kTcTileBytes / 16)),
-                 idesc_pv, (it > 0 || j > 0) ? 1u : 0u);
-        tc_commit(empty0 + 8 * s);            // the stage may be refilled once these MMAs have read it
-        tc_commit(bar_pv + 8 * (it & 1));     // P buffer free again, O updated
+      const int s = it % kTcStages;
+      const uint32_t stage = ring + s * kTcStageBytes;
+      const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
+      // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page, V read MN-major
+      const uint32_t pa0 = u_tmem + kTmemP + 32 * (it & 1);
+      const uint64_t vd0 = tc_desc(stage + kTcKBytes, kPageSize * 128, 1024);  // LBO: next 64 columns of d, SBO: next 8 tokens
+      // and l += P[:, 16j .. 16j+16) . 1 : the row sums of exactly the P that multiplies V
+      auto pv_page = [&](int j) {
+        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+        tc_mma_ts_if(leader, u_tmem + kTmemO, pa0 + 8 * j, vd0 + static_cast<uint64_t>(j * (kTcTileBytes / 16)), idesc_pv, acc);
+        tc_mma_ts_if(leader, u_tmem + kTmemL, pa0 + 8 * j, ones_desc, idesc_l, acc);
+      };
+      if (n_here == kTcPagesPerIter) {
+#pragma unroll
+        for (int j = 0; j < kTcPagesPerIter; ++j) pv_page(j);
+      } else {
+        for (int j = 0; j < n_here; ++j) pv_page(j);
       }
-      __syncwarp();
+      tc_commit_if(leader, empty0 + 8 * s);         // the stage may be refilled once these MMAs have read it
+      tc_commit_if(leader, bar_pv + 8 * (it & 1));  // O updated
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   } else {
@@ -310,11 +387,10 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int lim = mp.causal ? min(L, L - T + i_tok + 1) : L;
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;  // this warp's TMEM lanes
     const float scale_log2 = p.scale * 1.4426950408889634f;
-    float m_ref = -INFINITY;   // reference max the accumulated O and l are scaled by
-    float l = 0.f;
+    float m_ref = -INFINITY;   // reference max the accumulated O and l (both in tensor memory) are scaled by
     bool alive = true;
     for (int it = 0; it < n_iters && alive; ++it) {
-      bool ok = mbar_wait_bounded(bar_s + 8 * (it & 1), (it >> 1) & 1);
+      bool ok = mbar_spin_bounded(bar_s + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
       tc_fence_after();
@@ -324,68 +400,63 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       tmem_wait_ld();
       const int tok0 = (page0 + it * kTcPagesPerIter) * kPageSize;
       const int n_vis = min(lim, t1) - tok0;  // visible columns of this row in this iteration (may be <= 0)
-      float mx = -INFINITY;
+      if (__any_sync(0xffffffffu, n_vis < kTcPagesPerIter * kPageSize)) {  // boundary tiles only
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            sv[h][j] = (h * 32 + j < n_vis) ? sv[h][j] : 0xff800000u;  // -inf
+      }
+      // row maximum of the raw scores (the scale is positive), four independent chains
+      float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          float x = __uint_as_float(sv[h][j]) * scale_log2;
-          x = (h * 32 + j < n_vis) ? x : -INFINITY;
-          sv[h][j] = __float_as_uint(x);
-          mx = fmaxf(mx, x);
-        }
+        for (int j = 0; j < 32; ++j) mxs[j & 3] = fmaxf(mxs[j & 3], __uint_as_float(sv[h][j]));
+      const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * scale_log2;
       // lazy rescaling: keep the old reference unless the max grew past the threshold
       float m_new = m_ref;
       if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = fmaxf(m_ref, mx);
       const bool need = m_new != m_ref && m_ref != -INFINITY;
-      if (it >= 2) {  // PV(it-2) has finished reading the P buffer this iteration writes
-        ok = mbar_wait_bounded(bar_pv + 8 * (it & 1), ((it >> 1) - 1) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
-      }
+      // The P buffer this iteration writes is free: PV(it-2) was issued before S(it), the tensor core
+      // completes its work in issue order, and bar_s(it) has been observed.
       if (it > 0) {
         if (__any_sync(0xffffffffu, need)) {
           // O may only be touched once PV(it-1) has completed (PV(it) is not issued before this
           // warp arrives on bar_p below)
-          ok = mbar_wait_bounded(bar_pv + 8 * ((it - 1) & 1), ((it - 1) >> 1) & 1);
+          ok = mbar_spin_bounded(bar_pv + 8 * ((it - 1) & 1), ((it - 1) >> 1) & 1);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
           tc_fence_after();
           const float alpha = need ? ex2(m_ref - m_new) : 1.f;
-          l *= alpha;
 #pragma unroll
-          for (int cb = 0; cb < D / 32; ++cb) {
+          for (int cb = 0; cb < D / 32 + 1; ++cb) {  // O, then the block of columns that holds l
             uint32_t ov[32];
-            tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
+            tmem_ld32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
-            tmem_st32(tmem_o + lane_base + 32 * cb, ov);
+            tmem_st32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
           }
           tmem_wait_st();
         }
       }
       m_ref = m_new;
       const float ref = m_ref == -INFINITY ? 0.f : m_ref;
-      // P = exp2(S - ref) as bf16 into row `tid` of the swizzled [128 rows][128 B] tile
-      float lsum = 0.f;
-      const uint32_t prow = smem_u32(p_smem) + (it & 1) * kTcPBytes + tid * 128;
+      // P = exp2(S - ref) as bf16 pairs into TMEM lane `tid`: the A operand of O += P . V
+      // (s * scale_log2 - ref by one packed FMA per two elements; masked columns stay -inf -> 0)
+      const uint64_t c2 = f32x2(__float_as_uint(scale_log2), __float_as_uint(scale_log2));
+      const uint64_t nr2 = f32x2(__float_as_uint(-ref), __float_as_uint(-ref));
+      uint32_t pw[32];
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int j = ch * 8 + 2 * e;
-          const float p0 = ex2(__uint_as_float(sv[j >> 5][j & 31]) - ref);
-          const float p1 = ex2(__uint_as_float(sv[(j + 1) >> 5][(j + 1) & 31]) - ref);
-          lsum += p0 + p1;
-          w[e] = pack2<false>(p0, p1);
-        }
-        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};"
-                     ::"r"(prow + ((ch ^ (tid & 7)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]));
+      for (int j = 0; j < 32; ++j) {
+        const uint64_t x2 = fma_f32x2(f32x2(sv[j >> 4][(2 * j) & 31], sv[j >> 4][(2 * j + 1) & 31]), c2, nr2);
+        float x0, x1;
+        f32x2_split(x2, x0, x1);
+        pw[j] = pack2<false>(ex2(x0), ex2(x1));
       }
-      l += lsum;
-      fence_proxy_async();
+      tmem_st32(tmem_p + 32 * (it & 1) + lane_base, pw);
+      tmem_wait_st();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_tc(bar_p + 8 * (it & 1));
@@ -404,6 +475,13 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int dev_err = max(err, *cta_err);
     if (dev_err && tid == 0) report(p.status, dev_err);
     const bool valid_row = r < rows_total;
+    float l = 0.f;
+    if (alive && ok && n_iters > 0) {  // warp-uniform
+      uint32_t lv[32];
+      tmem_ld32(tmem_base + kTmemL + lane_base, lv);
+      tmem_wait_ld();
+      l = __uint_as_float(lv[0]);
+    }
     const bool live = !dev_err && alive && ok && l > 0.f;
     const float inv = live ? 1.f / l : 0.f;
     const int64_t qrow = (static_cast<int64_t>(b) * T + i_tok) * p.num_q_heads + g * G + (r % G);
@@ -458,6 +536,7 @@ bool attention_mq_tc_supports(const MqParams& mp) {
   const AttnParams& p = mp.a;
   if (p.geom.dtype != PDA_BF16 || p.geom.head_dim != kTcD) return false;
   if (p.group < 1 || mp.n_q < 1 || p.geom.num_pages < 1) return false;
+  if (!(p.scale > 0.f) || !(p.scale < INFINITY)) return false;  // the row maximum is taken before scaling
   const int64_t rows = static_cast<int64_t>(mp.n_q) * p.group;
   return p.geom.num_kv_heads * ((rows + kTcRows - 1) / kTcRows) <= 65535;
 }
