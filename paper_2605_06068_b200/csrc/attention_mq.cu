@@ -95,6 +95,7 @@ attention_mq_kernel(const __grid_constant__ CUtensorMap k_map,
 
   if (warp == kConsumers) {
     // ================= producer warp =================
+    const uint32_t leader = elect_one();
     bool bad = false;
     int pg = 0;
     for (int i = 0; i < n_tiles; ++i) {
@@ -113,17 +114,17 @@ attention_mq_kernel(const __grid_constant__ CUtensorMap k_map,
       if (i >= kStages) ok = mbar_wait_bounded(empty0 + 8 * s, ((i / kStages) - 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
-      if (lane == 0) {
-        if (kFp8) {
-          stage_scales[2 * s] = p.k_scale[static_cast<int64_t>(page) * p.geom.num_kv_heads + g];
-          stage_scales[2 * s + 1] = p.v_scale[static_cast<int64_t>(page) * p.geom.num_kv_heads + g];
-        }
-        const uint32_t dst = ring + s * C::kStageBytes;
-        fence_proxy_async();
-        mbar_expect_tx(full0 + 8 * s, C::kStageBytes);
-        tma_load_5d(dst, &k_map, full0 + 8 * s, 0, 0, 0, g, page);
-        tma_load_5d(dst + C::kTileBytes, &v_map, full0 + 8 * s, 0, 0, 0, g, page);
+      if (kFp8 && lane == 0) {
+        stage_scales[2 * s] = p.k_scale[static_cast<int64_t>(page) * p.geom.num_kv_heads + g];
+        stage_scales[2 * s + 1] = p.v_scale[static_cast<int64_t>(page) * p.geom.num_kv_heads + g];
       }
+      __syncwarp();
+      const uint32_t dst = ring + s * C::kStageBytes;
+      fence_proxy_async();
+      // (the elected lane issues, predicated: see elect_one)
+      mbar_expect_tx_if(leader, full0 + 8 * s, C::kStageBytes);
+      tma_load_5d_if(leader, dst, &k_map, full0 + 8 * s, 0, g, page);
+      tma_load_5d_if(leader, dst + C::kTileBytes, &v_map, full0 + 8 * s, 0, g, page);
     }
     if (bad && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
   }

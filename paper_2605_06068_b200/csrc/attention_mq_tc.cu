@@ -18,19 +18,21 @@
 // that the 4 pages of an iteration stack to [line][64 tokens][128 B]) and MN-major for V (contraction
 // over the 16 tokens of a page), so no data is rearranged in shared memory.
 //
-// Warp roles (6 warps): 0-3 softmax (thread t <-> TMEM lane t <-> query row t), 4 TMA producer,
-// 5 MMA issue + TMEM allocation. The producer and MMA warps stay converged and issue through one
-// elected lane with predicated instructions and warp-uniform operands: issued from inside a divergent
-// branch, a TMA copy or an MMA cost 90-200 clocks each here and the issuing thread was the bottleneck;
-// this way they cost 25-35. S and P are double-buffered so that the tensor core computes S of
-// iteration i+1 while the softmax warps work on i:
-//   MMA warp:   S(0); then per iteration i: S(i+1) -> commit(bar_s[(i+1)&1]);
-//               wait bar_p[i&1] -> PV(i), l(i) -> commit(stage empty), commit(bar_pv[i&1])
-//   softmax:    wait bar_s[i&1] -> tcgen05.ld S -> mask (boundary tiles), row max of the raw scores
-//               -> (rarely, after waiting for PV(i-1)) rescale O and l in TMEM when the running max
-//               grew by more than 2^8 -> P = exp2(S * scale - ref) as bf16 pairs (packed f32x2 FMA,
-//               one exp2 per element: the 16/clock/SM exp2 unit bounds these warps) -> tcgen05.st P
-//               -> arrive(bar_p[i&1])
+// Warp roles (10 warps): 0-3 and 4-7 two softmax sets (TMEM lane t <-> query row t; set x takes the
+// iterations it with it % 2 == x, so each scheduler holds one warp of each set and one covers the
+// other's waits), 8 TMA producer, 9 MMA issue + TMEM allocation. The producer and MMA warps stay
+// converged and issue through one elected lane with predicated instructions and warp-uniform operands:
+// issued from inside a divergent branch, a TMA copy or an MMA cost 90-200 clocks each here and the
+// issuing thread was the bottleneck; this way they cost 25-35. S and P are double-buffered:
+//   MMA warp:   S(j) as soon as stage j has landed and softmax(j-2) has loaded S(j-2) into registers
+//               (bar_sfree), ahead of PV; wait bar_p[i&1] -> PV(i), l(i) -> commit(stage empty),
+//               commit(bar_pv[i&1])
+//   softmax:    wait bar_s[i&1] -> tcgen05.ld S -> arrive(bar_sfree) -> mask (boundary tiles), row max
+//               of the raw scores -> running max of iteration i-1 from the other set (bar_m, shared
+//               memory) -> publish the new one -> (rarely, after waiting for PV(i-1)) rescale O and l in
+//               TMEM when the max grew by more than 2^8 -> wait PV(i-2) (P buffer free) -> P =
+//               exp2(S * scale - ref) as bf16 pairs (packed f32x2 FMA, one exp2 per element) ->
+//               tcgen05.st P -> arrive(bar_p[i&1])
 // All mbarrier waits are bounded; TMEM is always released before the CTA exits.
 #include "common.cuh"
 #include "tma_ptx.cuh"
@@ -42,13 +44,16 @@ namespace {
 constexpr int kTcD = 128;               // head_dim
 constexpr int kTcRows = 128;            // query rows per CTA (UMMA M)
 constexpr int kTcPagesPerIter = 4;      // 64 tokens per iteration
-constexpr int kTcStages = 5;
+constexpr int kTcStages = 6;
 constexpr int kTcTileBytes = kPageSize * kTcD * 2;        // 4096: one K or V page tile
 constexpr int kTcKBytes = kTcPagesPerIter * kTcTileBytes;  // 16 KB: K of 4 pages as [2 lines][64 tokens][128 B]
 constexpr int kTcStageBytes = 2 * kTcKBytes;               // 32 KB: K block, then 4 V page tiles
 constexpr int kTcOnesBytes = 2048;                         // bf16 ones: B operand [16 tokens][16 columns] of the row-sum MMA
-constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcOnesBytes + 256 + 1024;
-constexpr int kTcThreads = 192;
+constexpr int kTcMBytes = 2 * kTcRows * 4;                 // running row maxima handed between the two softmax sets
+constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcOnesBytes + kTcMBytes + 256 + 1024;
+constexpr int kTcSoftmaxWarps = 8;      // two sets of 4: set x takes the iterations it with it % 2 == x
+constexpr int kTcProducerWarp = 8, kTcMmaWarp = 9;
+constexpr int kTcThreads = 320;
 // Tensor memory columns (32-bit each, 128 lanes = query rows): S buffers 0..63 and 64..127 (f32),
 // O 128..255 (f32), Q 256..319 (bf16 pairs along d), P buffers 320..351 and 352..383 (bf16 pairs
 // along tokens). Allocations are powers of two.
@@ -68,13 +73,6 @@ __device__ __forceinline__ void mbar_arrive_tc(uint32_t bar) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// The MMA warp stays converged: one elected lane (the same one every time) issues, the instruction is
-// predicated rather than branched around, so warp-uniform operands can stay in uniform registers.
-__device__ __forceinline__ uint32_t elect_one() {
-  uint32_t is_leader;
-  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(is_leader));
-  return is_leader;
-}
 // D[tmem] (+)= A[tmem] . B[smem descriptor]; accumulate == 0 overwrites D. A is read from tensor memory
 // (lane = row, 32-bit column = two consecutive k elements).
 __device__ __forceinline__ void tc_mma_ts_if(uint32_t leader, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
@@ -89,19 +87,6 @@ __device__ __forceinline__ void tc_commit_if(uint32_t leader, uint32_t bar) {
       "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %1, 0;\n\t"
       "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
       ::"r"(bar), "r"(leader) : "memory");
-}
-__device__ __forceinline__ void tma_load_5d_if(uint32_t leader, uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                               int c2, int c3, int c4) {
-  asm volatile(
-      "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %6, 0;\n\t"
-      "@pe cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {0, 0, %3, %4, %5}], [%2];\n\t}"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c2), "r"(c3), "r"(c4), "r"(leader) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx_if(uint32_t leader, uint32_t bar, uint32_t bytes) {
-  asm volatile(
-      "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %2, 0;\n\t"
-      "@pe mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(bar), "r"(bytes), "r"(leader) : "memory");
 }
 // Shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field.
 __device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -163,8 +148,10 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* ones_smem = smem + kTcStages * kTcStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes);  // full[], empty[], s[2], p[2], pv[2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 6);
+  float* m_sh = reinterpret_cast<float*>(ones_smem + kTcOnesBytes);        // [2][128]
+  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 10);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -211,6 +198,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t ring = smem_u32(smem);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
+  const uint32_t bar_sfree = bar_pv + 16, bar_m = bar_sfree + 16;
   for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads) reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;
   fence_proxy_async();  // read by the tensor core through the async proxy
   if (tid == 0) {
@@ -220,14 +208,16 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     }
     for (int k = 0; k < 2; ++k) {
       mbar_init(bar_s + 8 * k, 1);
-      mbar_init(bar_p + 8 * k, 4);   // one arrival per softmax warp
+      mbar_init(bar_p + 8 * k, 4);   // one arrival per warp of the softmax set that owns the iteration
       mbar_init(bar_pv + 8 * k, 1);
+      mbar_init(bar_sfree + 8 * k, 4);
+      mbar_init(bar_m + 8 * k, 4);
     }
     *cta_err = 0;
     fence_mbar_init();
     fence_proxy_async();
   }
-  if (warp == 5) {  // tensor memory for S and O; this warp also releases it
+  if (warp == kTcMmaWarp) {  // tensor memory; this warp also releases it
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -258,14 +248,10 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     }
     tmem_wait_st();
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
 
-  if (warp == 4) {
-    // ================= TMA producer =================
+  if (warp == kTcProducerWarp) {
+    // ================= TMA producer (does not wait for Q) =================
     const uint32_t leader = elect_one();
     const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
@@ -304,7 +290,13 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
     }
     if (bad && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
-  } else if (warp == 5) {
+  } else {
+    // Q is in tensor memory before the first MMA is issued (the producer does not take part)
+    tc_fence_before();
+    asm volatile("bar.sync 1, %0;" ::"n"(kTcThreads - 32) : "memory");
+    tc_fence_after();
+  }
+  if (warp == kTcMmaWarp) {
     // ================= MMA issue =================
     constexpr uint32_t idesc_s = tc_idesc(kTcPagesPerIter * kPageSize, false);
     constexpr uint32_t idesc_pv = tc_idesc(D, true);
@@ -316,12 +308,21 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     const int u_tail0 = __shfl_sync(0xffffffffu, L - page0 * kPageSize, 0);  // tokens from the first page to the end
-    // Waits for stage `it`, clears the rows past the sequence end in V, issues S(it) = Q . K^T
-    auto issue_s = [&](int it) -> bool {
+    // S(j) may be issued once its stage has landed and, for j >= 2, the softmax warps have loaded
+    // S(j-2), whose buffer it overwrites, into registers
+    auto s_ready = [&](int j) -> bool {
+      if (j >= 2 && !mbar_test_wait(bar_sfree + 8 * (j & 1), ((j - 2) >> 1) & 1)) return false;
+      return mbar_test_wait(full0 + 8 * (j % kTcStages), (j / kTcStages) & 1);
+    };
+    auto s_wait = [&](int j) -> bool {
+      bool ok = true;
+      if (j >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (j & 1), ((j - 2) >> 1) & 1);
+      if (ok) ok = mbar_wait_bounded(full0 + 8 * (j % kTcStages), (j / kTcStages) & 1);
+      return __all_sync(0xffffffffu, ok);
+    };
+    // Clears the rows past the sequence end in V of stage `it`, issues S(it) = Q . K^T
+    auto issue_s = [&](int it) {
       const int s = it % kTcStages;
-      bool ok = mbar_wait_bounded(full0 + 8 * s, (it / kTcStages) & 1);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) return false;
       const uint32_t stage = ring + s * kTcStageBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       const int tail = u_tail0 - (it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
@@ -346,14 +347,19 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         tc_mma_ts_if(leader, d, u_tmem + kTmemQ + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
       }
       tc_commit_if(leader, bar_s + 8 * (it & 1));
-      return true;
     };
-    bool ok = u_iters > 0 ? issue_s(0) : true;
+    // S runs ahead of PV as far as its operands allow (the tensor core works in issue order, so S(it+1)
+    // should be in the queue before PV(it) waits for the softmax warps); only the S that PV(it) needs
+    // is waited for.
+    bool ok = true;
+    int next_s = 0;
     for (int it = 0; it < u_iters && ok; ++it) {
-      // S(it+1) goes to the other S buffer, which softmax(it-1) has released (it arrived on bar_p
-      // before PV(it-1) was issued)
-      if (it + 1 < u_iters) ok = issue_s(it + 1);
-      if (!ok) break;
+      while (next_s < u_iters && next_s <= it + 3 && s_ready(next_s)) issue_s(next_s++);
+      if (next_s <= it) {
+        ok = s_wait(next_s);
+        if (!ok) break;
+        issue_s(next_s++);
+      }
       ok = mbar_wait_bounded(bar_p + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -377,27 +383,37 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         for (int j = 0; j < n_here; ++j) pv_page(j);
       }
       tc_commit_if(leader, empty0 + 8 * s);         // the stage may be refilled once these MMAs have read it
-      tc_commit_if(leader, bar_pv + 8 * (it & 1));  // O updated
+      tc_commit_if(leader, bar_pv + 8 * (it & 1));  // O and l updated, P buffer free again
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
-  } else {
-    // ================= softmax: thread t owns query row t =================
-    const int r = rb * kTcRows + tid;
+  } else if (warp < kTcSoftmaxWarps) {
+    // ================= softmax: TMEM lane t <-> query row t; set x takes iterations x, x+2, ... ==========
+    // Two warps per scheduler, one of each set: while one waits (for S, for the other set's row maximum,
+    // for its tcgen05.ld/st) the other keeps the exp2 unit busy, which is what bounds this part.
+    const int set = warp >> 2, t = tid & (kTcRows - 1);
+    const int r = rb * kTcRows + t;
     const int i_tok = r / G;
     const int lim = mp.causal ? min(L, L - T + i_tok + 1) : L;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;  // this warp's TMEM lanes
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;  // this warp's TMEM lanes
     const float scale_log2 = p.scale * 1.4426950408889634f;
+    const uint32_t my_s = bar_s + 8 * set, my_p = bar_p + 8 * set, my_pv = bar_pv + 8 * set;
+    const uint32_t my_sfree = bar_sfree + 8 * set, my_m = bar_m + 8 * set, other_m = bar_m + 8 * (set ^ 1);
     float m_ref = -INFINITY;   // reference max the accumulated O and l (both in tensor memory) are scaled by
     bool alive = true;
-    for (int it = 0; it < n_iters && alive; ++it) {
-      bool ok = mbar_spin_bounded(bar_s + 8 * (it & 1), (it >> 1) & 1);
+    auto fail = [&]() { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; };
+    for (int it = set; it < n_iters; it += 2) {
+      const int k = it >> 1;  // this set's k-th iteration: the phase index of its barriers
+      bool ok = mbar_spin_bounded(my_s, k & 1);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
+      if (!ok) { fail(); break; }
       tc_fence_after();
       uint32_t sv[2][32];
-      tmem_ld32(tmem_s + 64 * (it & 1) + lane_base, sv[0]);
-      tmem_ld32(tmem_s + 64 * (it & 1) + lane_base + 32, sv[1]);
+      tmem_ld32(tmem_s + 64 * set + lane_base, sv[0]);
+      tmem_ld32(tmem_s + 64 * set + lane_base + 32, sv[1]);
       tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_tc(my_sfree);  // S(it) is in registers: S(it+2) may overwrite its buffer
       const int tok0 = (page0 + it * kTcPagesPerIter) * kPageSize;
       const int n_vis = min(lim, t1) - tok0;  // visible columns of this row in this iteration (may be <= 0)
       if (__any_sync(0xffffffffu, n_vis < kTcPagesPerIter * kPageSize)) {  // boundary tiles only
@@ -414,37 +430,48 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
         for (int j = 0; j < 32; ++j) mxs[j & 3] = fmaxf(mxs[j & 3], __uint_as_float(sv[h][j]));
       const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * scale_log2;
+      // the reference after iteration it-1 comes from the other set
+      if (it > 0) {
+        ok = mbar_spin_bounded(other_m, ((it - 1) >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { fail(); break; }
+        m_ref = m_sh[((it - 1) & 1) * kTcRows + t];
+      }
       // lazy rescaling: keep the old reference unless the max grew past the threshold
       float m_new = m_ref;
       if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = fmaxf(m_ref, mx);
       const bool need = m_new != m_ref && m_ref != -INFINITY;
-      // The P buffer this iteration writes is free: PV(it-2) was issued before S(it), the tensor core
-      // completes its work in issue order, and bar_s(it) has been observed.
-      if (it > 0) {
-        if (__any_sync(0xffffffffu, need)) {
-          // O may only be touched once PV(it-1) has completed (PV(it) is not issued before this
-          // warp arrives on bar_p below)
-          ok = mbar_spin_bounded(bar_pv + 8 * ((it - 1) & 1), ((it - 1) >> 1) & 1);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; break; }
-          tc_fence_after();
-          const float alpha = need ? ex2(m_ref - m_new) : 1.f;
+      m_sh[(it & 1) * kTcRows + t] = m_new;
+      __syncwarp();
+      if (lane == 0) mbar_arrive_tc(my_m);  // (release: the other set reads m_sh after its wait)
+      if (it >= 2) {  // PV(it-2) has finished reading the P buffer this iteration writes
+        ok = mbar_spin_bounded(my_pv, (k - 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { fail(); break; }
+      }
+      if (it > 0 && __any_sync(0xffffffffu, need)) {
+        // O and l may only be touched once PV(it-1) has completed; PV(it) is not issued before this
+        // warp arrives on bar_p below, and the other set rescales only after PV(it)
+        ok = mbar_spin_bounded(bar_pv + 8 * (set ^ 1), ((it - 1) >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { fail(); break; }
+        tc_fence_after();
+        const float alpha = need ? ex2(m_ref - m_new) : 1.f;
 #pragma unroll
-          for (int cb = 0; cb < D / 32 + 1; ++cb) {  // O, then the block of columns that holds l
-            uint32_t ov[32];
-            tmem_ld32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
-            tmem_wait_ld();
+        for (int cb = 0; cb < D / 32 + 1; ++cb) {  // O, then the block of columns that holds l
+          uint32_t ov[32];
+          tmem_ld32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
+          tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
-            tmem_st32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
-          }
-          tmem_wait_st();
+          for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
+          tmem_st32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
         }
+        tmem_wait_st();
       }
       m_ref = m_new;
       const float ref = m_ref == -INFINITY ? 0.f : m_ref;
-      // P = exp2(S - ref) as bf16 pairs into TMEM lane `tid`: the A operand of O += P . V
-      // (s * scale_log2 - ref by one packed FMA per two elements; masked columns stay -inf -> 0)
+      // P = exp2(S * scale_log2 - ref) as bf16 pairs into TMEM lane t: the A operand of O += P . V
+      // (one packed FMA per two elements; masked columns stay -inf -> 0)
       const uint64_t c2 = f32x2(__float_as_uint(scale_log2), __float_as_uint(scale_log2));
       const uint64_t nr2 = f32x2(__float_as_uint(-ref), __float_as_uint(-ref));
       uint32_t pw[32];
@@ -455,41 +482,51 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         f32x2_split(x2, x0, x1);
         pw[j] = pack2<false>(ex2(x0), ex2(x1));
       }
-      tmem_st32(tmem_p + 32 * (it & 1) + lane_base, pw);
+      tmem_st32(tmem_p + 32 * set + lane_base, pw);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_tc(bar_p + 8 * (it & 1));
+      if (lane == 0) mbar_arrive_tc(my_p);
     }
 
-    // ---- finalise this row
-    bool ok = true;
+    // ---- finalise: the last iteration's reference (from the set that owned it) and the last PV
+    bool ok = alive;
     if (alive && n_iters > 0) {
-      ok = mbar_wait_bounded(bar_pv + 8 * ((n_iters - 1) & 1), ((n_iters - 1) >> 1) & 1);
-      ok = __all_sync(0xffffffffu, ok);
+      const int last = n_iters - 1;
+      if ((last & 1) != set) {
+        ok = mbar_spin_bounded(bar_m + 8 * (last & 1), (last >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) m_ref = m_sh[(last & 1) * kTcRows + t];
+      }
+      if (ok) {
+        ok = mbar_wait_bounded(bar_pv + 8 * (last & 1), (last >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+      }
       if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
       tc_fence_after();
     }
     // every softmax warp reaches this point together with its error view settled
-    asm volatile("bar.sync 1, 128;" ::: "memory");
+    asm volatile("bar.sync 2, %0;" ::"n"(kTcSoftmaxWarps * 32) : "memory");
     const int dev_err = max(err, *cta_err);
     if (dev_err && tid == 0) report(p.status, dev_err);
     const bool valid_row = r < rows_total;
+    const bool have = alive && ok && n_iters > 0;  // warp-uniform
     float l = 0.f;
-    if (alive && ok && n_iters > 0) {  // warp-uniform
+    if (have) {
       uint32_t lv[32];
       tmem_ld32(tmem_base + kTmemL + lane_base, lv);
       tmem_wait_ld();
       l = __uint_as_float(lv[0]);
     }
-    const bool live = !dev_err && alive && ok && l > 0.f;
+    const bool live = !dev_err && have && l > 0.f;
     const float inv = live ? 1.f / l : 0.f;
     const int64_t qrow = (static_cast<int64_t>(b) * T + i_tok) * p.num_q_heads + g * G + (r % G);
     constexpr float kLn2 = 0.6931471805599453f;
+    // set x stores columns [64 x, 64 x + 64) of the row
 #pragma unroll
-    for (int cb = 0; cb < D / 32; ++cb) {
+    for (int cb = 2 * set; cb < 2 * set + 2; ++cb) {
       uint32_t ov[32];
-      if (alive && ok && n_iters > 0) {  // warp-uniform
+      if (have) {
         tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
         tmem_wait_ld();
       } else {
@@ -517,14 +554,14 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         }
       }
     }
-    if (split && valid_row)
+    if (split && valid_row && set == 0)
       p.part_lse[qrow * p.max_chunks + p.chunk_slot0 + c] = live ? (m_ref + __log2f(l)) * kLn2 : -INFINITY;
   }
 
   // ---- teardown: everyone is done with tensor memory before it is released
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kTcMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }

@@ -122,13 +122,14 @@ attention_persist_kernel(const __grid_constant__ CUtensorMap k_map,
       }
     }
   };
-  auto issue = [&](uint32_t ordinal, int g, int page_raw) {  // lane 0 only
+  const uint32_t leader = elect_one();
+  auto issue = [&](uint32_t ordinal, int g, int page_raw) {  // whole warp, converged; the elected lane issues
     const int s = ordinal % kStages;
     const uint32_t bar = bar0 + 8 * s;
     const uint32_t dst = ring + s * C::kStageBytes;
-    mbar_expect_tx(bar, C::kStageBytes);
-    tma_load_5d(dst, &k_map, bar, 0, 0, 0, g, max(page_raw, 0));
-    tma_load_5d(dst + C::kTileBytes, &v_map, bar, 0, 0, 0, g, max(page_raw, 0));
+    mbar_expect_tx_if(leader, bar, C::kStageBytes);
+    tma_load_5d_if(leader, dst, &k_map, bar, 0, g, max(page_raw, 0));
+    tma_load_5d_if(leader, dst + C::kTileBytes, &v_map, bar, 0, g, max(page_raw, 0));
   };
 
   const float scale_log2 = p.scale * 1.4426950408889634f;
@@ -142,7 +143,7 @@ attention_persist_kernel(const __grid_constant__ CUtensorMap k_map,
   for (int j = 0; j < min(kStages, n_mine); ++j) {
     const int page = __shfl_sync(0xffffffffu, pgA, j);
     if (page < 0) bad_page = true;
-    if (lane == 0) issue(ord + j, cur.g, page);
+    issue(ord + j, cur.g, page);
   }
 
   // Q^T fragments of the current unit and, once its ticket is known, of the next one
@@ -247,10 +248,8 @@ attention_persist_kernel(const __grid_constant__ CUtensorMap k_map,
         if ((kn >> 5) == ((kk + 1) >> 5)) page = __shfl_sync(0xffffffffu, pgA, kn & 31);
         else page = __shfl_sync(0xffffffffu, pgB, kn & 31);
         if (page < 0) bad_page = true;
-        if (lane == 0) {
-          fence_proxy_async();
-          issue(ord + kn, cur.g, page);
-        }
+        fence_proxy_async();
+        issue(ord + kn, cur.g, page);
       }
     }
 

@@ -149,14 +149,15 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
   load_block(0, pgA, ksA, vsA);
   load_block(1, pgB, ksB, vsB);
 
-  auto issue = [&](int kk, int page_raw) {  // lane 0 only
+  const uint32_t leader = elect_one();
+  auto issue = [&](int kk, int page_raw) {  // whole warp, converged; the elected lane issues
     const int page = max(page_raw, 0);
     const int s = kk % kStages;
     const uint32_t bar = bar0 + 8 * s;
     const uint32_t dst = ring + s * C::kStageBytes;
-    mbar_expect_tx(bar, C::kStageBytes);
-    tma_load_5d(dst, &k_map, bar, 0, 0, 0, g, page);
-    tma_load_5d(dst + C::kTileBytes, &v_map, bar, 0, 0, 0, g, page);
+    mbar_expect_tx_if(leader, bar, C::kStageBytes);
+    tma_load_5d_if(leader, dst, &k_map, bar, 0, g, page);
+    tma_load_5d_if(leader, dst + C::kTileBytes, &v_map, bar, 0, g, page);
   };
 
   // prologue: fill the ring
@@ -165,7 +166,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     for (int kk = 0; kk < n_pre; ++kk) {
       const int page = __shfl_sync(0xffffffffu, pgA, kk);
       if (page < 0) bad_page = true;
-      if (lane == 0) issue(kk, page);
+      issue(kk, page);
     }
   }
   const bool append_here = sp.k_new != nullptr && !err && L > 0 && c == nch - 1;
@@ -246,10 +247,8 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       const bool in_a = (kn >> 5) == ((kk + 1) >> 5);
       const int page = __shfl_sync(0xffffffffu, in_a ? pgA : pgB, kn & 31);
       if (page < 0) bad_page = true;
-      if (lane == 0) {
-        fence_proxy_async();
-        issue(kn, page);
-      }
+      fence_proxy_async();
+      issue(kn, page);
     }
   }
 
