@@ -18,15 +18,17 @@
 // that the 4 pages of an iteration stack to [line][64 tokens][128 B]) and MN-major for V (contraction
 // over the 16 tokens of a page), so no data is rearranged in shared memory.
 //
-// Warp roles (10 warps): 0-3 and 4-7 two softmax sets (TMEM lane t <-> query row t; set x takes the
+// Warp roles (11 warps): 0-3 and 4-7 two softmax sets (TMEM lane t <-> query row t; set x takes the
 // iterations it with it % 2 == x, so each scheduler holds one warp of each set and one covers the
-// other's waits), 8 TMA producer, 9 MMA issue + TMEM allocation. The producer and MMA warps stay
+// other's waits), 8 TMA producer, 9 S issue + TMEM allocation, 10 PV issue (one issuing warp for both was
+// measured to be the bottleneck: a few hundred dependent scalar instructions per iteration at one every
+// 4-8 clocks). The producer and issuing warps stay
 // converged and issue through one elected lane with predicated instructions and warp-uniform operands:
 // issued from inside a divergent branch, a TMA copy or an MMA cost 90-200 clocks each here and the
 // issuing thread was the bottleneck; this way they cost 25-35. S and P are double-buffered:
-//   MMA warp:   S(j) as soon as stage j has landed and softmax(j-2) has loaded S(j-2) into registers
-//               (bar_sfree), ahead of PV; wait bar_p[i&1] -> PV(i), l(i) -> commit(stage empty),
-//               commit(bar_pv[i&1])
+//   S warp:     S(j) as soon as stage j has landed and softmax(j-2) has loaded S(j-2) into registers
+//               (bar_sfree) -> commit(bar_s[j&1])
+//   PV warp:    wait bar_p[i&1] -> PV(i), l(i) -> commit(stage empty), commit(bar_pv[i&1])
 //   softmax:    wait bar_s[i&1] -> tcgen05.ld S -> arrive(bar_sfree) -> mask (boundary tiles), row max
 //               of the raw scores -> running max of iteration i-1 from the other set (bar_m, shared
 //               memory) -> publish the new one -> (rarely, after waiting for PV(i-1)) rescale O and l in
@@ -52,8 +54,8 @@ constexpr int kTcOnesBytes = 2048;                         // bf16 ones: B opera
 constexpr int kTcMBytes = 2 * kTcRows * 4;                 // running row maxima handed between the two softmax sets
 constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcOnesBytes + kTcMBytes + 256 + 1024;
 constexpr int kTcSoftmaxWarps = 8;      // two sets of 4: set x takes the iterations it with it % 2 == x
-constexpr int kTcProducerWarp = 8, kTcMmaWarp = 9;
-constexpr int kTcThreads = 320;
+constexpr int kTcProducerWarp = 8, kTcMmaWarp = 9, kTcPvWarp = 10;  // (the MMA warp issues S and owns the TMEM allocation)
+constexpr int kTcThreads = 352;
 // Tensor memory columns (32-bit each, 128 lanes = query rows): S buffers 0..63 and 64..127 (f32),
 // O 128..255 (f32), Q 256..319 (bf16 pairs along d), P buffers 320..351 and 352..383 (bf16 pairs
 // along tokens). Allocations are powers of two.
@@ -297,36 +299,30 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     tc_fence_after();
   }
   if (warp == kTcMmaWarp) {
-    // ================= MMA issue =================
+    // ================= S issue: S(it) = Q . K^T as soon as its operands allow =================
+    // (Two issuing warps, one for S and one for PV: a single warp runs the few hundred dependent scalar
+    // instructions of both per iteration at one every 4-8 clocks, which is as long as the iteration
+    // itself. Each keeps to its own chain of barriers; the tensor core's order between the two does not
+    // matter.)
     constexpr uint32_t idesc_s = tc_idesc(kTcPagesPerIter * kPageSize, false);
-    constexpr uint32_t idesc_pv = tc_idesc(D, true);
-    constexpr uint32_t idesc_l = tc_idesc(16, false);
-    const uint64_t ones_desc = tc_desc(smem_u32(ones_smem), 16, 1024);
     const uint32_t leader = elect_one();
     // warp-uniform copies (a shuffle from lane 0 tells the compiler so)
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
     const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     const int u_tail0 = __shfl_sync(0xffffffffu, L - page0 * kPageSize, 0);  // tokens from the first page to the end
-    // S(j) may be issued once its stage has landed and, for j >= 2, the softmax warps have loaded
-    // S(j-2), whose buffer it overwrites, into registers
-    auto s_ready = [&](int j) -> bool {
-      if (j >= 2 && !mbar_test_wait(bar_sfree + 8 * (j & 1), ((j - 2) >> 1) & 1)) return false;
-      return mbar_test_wait(full0 + 8 * (j % kTcStages), (j / kTcStages) & 1);
-    };
-    auto s_wait = [&](int j) -> bool {
-      bool ok = true;
-      if (j >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (j & 1), ((j - 2) >> 1) & 1);
-      if (ok) ok = mbar_wait_bounded(full0 + 8 * (j % kTcStages), (j / kTcStages) & 1);
-      return __all_sync(0xffffffffu, ok);
-    };
-    // Clears the rows past the sequence end in V of stage `it`, issues S(it) = Q . K^T
-    auto issue_s = [&](int it) {
-      const int s = it % kTcStages;
-      const uint32_t stage = ring + s * kTcStageBytes;
+    bool ok = true;
+    uint32_t stage_i = 0, stage_par = 0;  // the iteration's ring stage and that stage's phase parity
+    for (int it = 0; it < u_iters; ++it) {
+      // S(it) overwrites the buffer of S(it-2): the softmax warps have loaded that into registers
+      if (it >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (it & 1), ((it - 2) >> 1) & 1);
+      if (ok) ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);  // the stage has landed
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const uint32_t stage = ring + stage_i * kTcStageBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       const int tail = u_tail0 - (it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
-      if (tail < kPageSize) {
+      if (tail < kPageSize) {  // clear the rows past the sequence end in V (P is 0 there, V must be finite)
         const uint32_t vt = stage + kTcKBytes + (n_here - 1) * kTcTileBytes;
         for (int i = lane; i < (kPageSize - tail) * 16; i += 32) {
           const int r = tail + i / 16, ch = i % 16;
@@ -347,25 +343,26 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         tc_mma_ts_if(leader, d, u_tmem + kTmemQ + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
       }
       tc_commit_if(leader, bar_s + 8 * (it & 1));
-    };
-    // S runs ahead of PV as far as its operands allow (the tensor core works in issue order, so S(it+1)
-    // should be in the queue before PV(it) waits for the softmax warps); only the S that PV(it) needs
-    // is waited for.
+      if (++stage_i == kTcStages) { stage_i = 0; stage_par ^= 1; }
+    }
+    if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
+  } else if (warp == kTcPvWarp) {
+    // ================= PV issue: O += P . V and l += P . 1 =================
+    constexpr uint32_t idesc_pv = tc_idesc(D, true);
+    constexpr uint32_t idesc_l = tc_idesc(16, false);
+    const uint64_t ones_desc = tc_desc(smem_u32(ones_smem), 16, 1024);
+    const uint32_t leader = elect_one();
+    const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
+    const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
+    const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     bool ok = true;
-    int next_s = 0;
-    for (int it = 0; it < u_iters && ok; ++it) {
-      while (next_s < u_iters && next_s <= it + 3 && s_ready(next_s)) issue_s(next_s++);
-      if (next_s <= it) {
-        ok = s_wait(next_s);
-        if (!ok) break;
-        issue_s(next_s++);
-      }
+    uint32_t stage_i = 0;
+    for (int it = 0; it < u_iters; ++it) {
       ok = mbar_wait_bounded(bar_p + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int s = it % kTcStages;
-      const uint32_t stage = ring + s * kTcStageBytes;
+      const uint32_t stage = ring + stage_i * kTcStageBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page, V read MN-major
       const uint32_t pa0 = u_tmem + kTmemP + 32 * (it & 1);
@@ -382,8 +379,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       } else {
         for (int j = 0; j < n_here; ++j) pv_page(j);
       }
-      tc_commit_if(leader, empty0 + 8 * s);         // the stage may be refilled once these MMAs have read it
-      tc_commit_if(leader, bar_pv + 8 * (it & 1));  // O and l updated, P buffer free again
+      tc_commit_if(leader, empty0 + 8 * stage_i);     // the stage may be refilled once these MMAs have read it
+      tc_commit_if(leader, bar_pv + 8 * (it & 1));    // O and l updated, P buffer free again
+      if (++stage_i == kTcStages) stage_i = 0;
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   } else if (warp < kTcSoftmaxWarps) {
