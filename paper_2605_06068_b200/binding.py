@@ -218,7 +218,9 @@ def paged_decode_step_host(q_host, k_new_host, v_new_host, block_table_host, seq
                            q_dev, k_new_dev, v_new_dev, block_table_dev, seq_lens_dev,
                            k_cache, v_cache, scale, chunk_tokens, part_o, part_lse,
                            out_dev, out_host, workspace=None, status=None, stream=None):
-    """Fused decode step from pinned host inputs to a host output."""
+    """Fused decode step from pinned host inputs to a host output. ``q_dev``, ``k_new_dev``,
+    ``v_new_dev`` and ``out_dev`` may be None: the kernel then works on the pinned host buffers in
+    place (see ``include/pda.h``)."""
     desc = cache_desc(k_cache)
     B, Hq, _ = q_host.shape
     mc = 0 if part_o is None else part_o.shape[2]

@@ -90,6 +90,21 @@ int check_attention(const void* q, const void* k_cache, const void* v_cache,
 
 }  // namespace
 
+namespace {
+// Device address of pinned, mapped host memory (what cudaHostAlloc / cudaHostRegister give); NULL for
+// anything the device cannot reach.
+void* mapped_device_pointer(const void* host) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  if (a.type != cudaMemoryTypeHost && a.type != cudaMemoryTypeManaged && a.type != cudaMemoryTypeDevice)
+    return nullptr;
+  return a.devicePointer;
+}
+}  // namespace
+
 extern "C" {
 
 int pda_version(void) { return PDA_VERSION; }
@@ -386,24 +401,32 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
                            int32_t max_chunks, int32_t* workspace, void* out_dev, void* out_host,
                            int32_t* status, pda_stream_t stream) {
   AttnParams p;
-  if (!out_dev || !out_host) return PDA_ERR_INVALID_ARG;
-  if (int rc = check_attention(q_dev, k_cache, v_cache, desc, nullptr, nullptr, block_table_dev,
+  if (!out_host || !q_host || !k_new_host || !v_new_host) return PDA_ERR_INVALID_ARG;
+  // A staging buffer that is NULL means "in place": the kernel reads (writes) the host buffer itself
+  // over the bus, which needs pinned, device-mapped host memory.
+  const void* q_use = q_dev;
+  const void* k_use = k_new_dev;
+  const void* v_use = v_new_dev;
+  void* out_use = out_dev;
+  if (!q_dev && !(q_use = mapped_device_pointer(q_host))) return PDA_ERR_INVALID_ARG;
+  if (!k_new_dev && !(k_use = mapped_device_pointer(k_new_host))) return PDA_ERR_INVALID_ARG;
+  if (!v_new_dev && !(v_use = mapped_device_pointer(v_new_host))) return PDA_ERR_INVALID_ARG;
+  if (!out_dev && !(out_use = mapped_device_pointer(out_host))) return PDA_ERR_INVALID_ARG;
+  if (int rc = check_attention(q_use, k_cache, v_cache, desc, nullptr, nullptr, block_table_dev,
                                block_table_stride, seq_lens_dev, batch, num_q_heads,
-                               chunk_tokens, out_dev, part_o, part_lse, max_chunks, &p))
+                               chunk_tokens, out_use, part_o, part_lse, max_chunks, &p))
     return rc;
   if (p.geom.dtype != PDA_BF16) return PDA_ERR_UNSUPPORTED;
   if (batch == 0) return PDA_OK;
-  if (!q_host || !k_new_host || !v_new_host || !block_table_host || !seq_lens_host ||
-      !k_new_dev || !v_new_dev)
-    return PDA_ERR_INVALID_ARG;
+  if (!block_table_host || !seq_lens_host) return PDA_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t D = p.geom.head_dim;
   const size_t q_bytes = static_cast<size_t>(batch) * num_q_heads * D * 2;
   const size_t new_bytes = static_cast<size_t>(batch) * p.geom.num_kv_heads * D * 2;
   cudaError_t e;
-  if ((e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, s))) return e;
-  if ((e = cudaMemcpyAsync(k_new_dev, k_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
-  if ((e = cudaMemcpyAsync(v_new_dev, v_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
+  if (q_dev && (e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, s))) return e;
+  if (k_new_dev && (e = cudaMemcpyAsync(k_new_dev, k_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
+  if (v_new_dev && (e = cudaMemcpyAsync(v_new_dev, v_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
   if ((e = cudaMemcpyAsync(block_table_dev, block_table_host,
                            static_cast<size_t>(batch) * block_table_stride * 4,
                            cudaMemcpyHostToDevice, s)))
@@ -411,12 +434,12 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
   if ((e = cudaMemcpyAsync(seq_lens_dev, seq_lens_host, static_cast<size_t>(batch) * 4,
                            cudaMemcpyHostToDevice, s)))
     return e;
-  if (int rc = paged_decode_step(q_dev, k_new_dev, v_new_dev, k_cache, v_cache, desc, nullptr, nullptr,
+  if (int rc = paged_decode_step(q_use, k_use, v_use, k_cache, v_cache, desc, nullptr, nullptr,
                                  block_table_dev, block_table_stride, seq_lens_dev, batch,
-                                 num_q_heads, scale, chunk_tokens, out_dev, part_o, part_lse,
+                                 num_q_heads, scale, chunk_tokens, out_use, part_o, part_lse,
                                  max_chunks, workspace, status, stream))
     return rc;
-  if ((e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, s))) return e;
+  if (out_dev && (e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, s))) return e;
   return PDA_OK;
 }
 

@@ -451,6 +451,23 @@ def test_step_host_matches_device_calls(oracle):
         assert_close(got, ref, what=f"step_host chunk {chunk}")
         k_ref, _ = host_appended(oracle, w)
         assert (bf16_to_bits(dw.k_cache) == k_ref).all()
+        # in place: no staging buffers, the kernel reads q / k_new / v_new from and writes the result to
+        # the pinned (device-mapped) host buffers; same result, and a plain (unmapped) buffer is refused
+        dw = DeviceWorkload(w)
+        out_host2 = torch.zeros(w.q.shape, dtype=torch.int16).pin_memory()
+        pda.paged_decode_step_host(hq.view(torch.bfloat16), hk, hv, hbt, hsl, None, None, None, dbt, dsl,
+                                   dw.k_cache, dw.v_cache, float(w.scale), chunk, po, pl,
+                                   None, out_host2, workspace=pda.new_workspace(w.batch, 8),
+                                   status=dw.status)
+        torch.cuda.synchronize()
+        got2 = W.bf16_bits_to_f32(out_host2.numpy().view(np.uint16)).astype(np.float64)
+        assert_close(got2, ref, what=f"step_host in place chunk {chunk}")
+        assert (bf16_to_bits(dw.k_cache) == k_ref).all()
+        assert int(dw.status.item()) == 0
+    with pytest.raises(RuntimeError):
+        pda.paged_decode_step_host(hq.view(torch.bfloat16), hk, hv, hbt, hsl, None, None, None, dbt, dsl,
+                                   dw.k_cache, dw.v_cache, float(w.scale), 0, None, None,
+                                   None, torch.zeros(w.q.shape, dtype=torch.int16), status=dw.status)
 
 
 # ---- sliding window -------------------------------------------------------------------------
