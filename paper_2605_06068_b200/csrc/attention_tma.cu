@@ -333,6 +333,51 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     __syncthreads();
     if (cta_err[1]) {
       __threadfence();
+      // The merge is the tail of the unit (and, for the last unit, of the launch), so it is spread over
+      // the whole CTA with every load independent of the others: a warp per head turns the chunks'
+      // log-sum-exps into weights in shared memory (the TMA rings are idle by now), then a thread per
+      // (head, 4 columns) accumulates the chunks' partial rows with 16-byte loads.
+      float* w_sh = reinterpret_cast<float*>(smem);  // [G][nch] weights, then [G] 1 / sum
+      const bool fits = static_cast<int64_t>(G) * (nch + 1) * 4 <= static_cast<int64_t>(kWarps) * C::kWarpRing;
+      if (fits) {
+        for (int h = warp; h < G; h += kWarps) {
+          const float* lse = p.part_lse + (row0 + h) * p.max_chunks + p.chunk_slot0;
+          float M = -INFINITY;
+          for (int cc = lane; cc < nch; cc += 32) M = fmaxf(M, __ldcg(lse + cc));
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+          float W = 0.f;
+          for (int cc = lane; cc < nch; cc += 32) {
+            const float w = M > -INFINITY ? __expf(__ldcg(lse + cc) - M) : 0.f;
+            w_sh[h * nch + cc] = w;
+            W += w;
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) W += __shfl_xor_sync(0xffffffffu, W, o);
+          if (lane == 0) w_sh[G * nch + h] = W > 0.f ? 1.f / W : 0.f;
+        }
+        __syncthreads();
+        constexpr int kVec = D / 4;
+        for (int idx = tid; idx < G * kVec; idx += kWarps * 32) {
+          const int h = idx / kVec, d4 = idx % kVec;
+          const int64_t row = row0 + h;
+          const float4* po = reinterpret_cast<const float4*>(p.part_o + (row * p.max_chunks + p.chunk_slot0) * D) + d4;
+          const float* wh = w_sh + h * nch;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+          for (int cc = 0; cc < nch; ++cc) {
+            const float4 v = __ldcg(po + static_cast<int64_t>(cc) * kVec);
+            const float w = wh[cc];
+            acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
+            acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+          }
+          const float inv = w_sh[G * nch + h];
+          uint2 packed;
+          packed.x = pack2<false>(acc.x * inv, acc.y * inv);
+          packed.y = pack2<false>(acc.z * inv, acc.w * inv);
+          *reinterpret_cast<uint2*>(p.out + row * D + 4 * d4) = packed;
+        }
+      } else {
       for (int idx = tid; idx < G * D; idx += kWarps * 32) {
         const int h = idx / D, d = idx % D;
         const int64_t row = row0 + h;
@@ -350,6 +395,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
           acc /= W;
         }
         p.out[row * D + d] = __float2bfloat16_rn(acc);
+      }
       }
       if (tid == 0) *counter = 0;  // leave the workspace clean for the next call
     }
