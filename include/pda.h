@@ -230,8 +230,13 @@ int paged_verify_attention(const void* q, const void* k_cache, const void* v_cac
  *                  with max_chunks >= ceil(prefix_tokens/prefix_chunk_tokens)
  *                                    + ceil((max seq_len - prefix_tokens)/chunk_tokens)
  *   out            [batch, num_q_heads, head_dim] bf16
- * Three launches on `stream` (prefix, suffixes, merge). Supported: group size <= 8,
- * head_dim 64/128 (bf16) or 128 (e4m3), batch <= 4096. */
+ * Three launches (prefix, suffixes, merge), ordered on `stream`; the suffix launch,
+ * which is independent of the prefix launch, runs beside it on a stream the
+ * library owns (forked from and joined back to `stream` with events, which is
+ * also valid while `stream` is being captured; the side stream is created by the
+ * first call that is not inside a capture, and until it exists the launches simply
+ * follow one another on `stream`). Supported: group size <= 8, head_dim 64/128
+ * (bf16) or 128 (e4m3), batch <= 4096. */
 int paged_prefix_decode_attention(const void* q, const void* k_cache, const void* v_cache,
                                   const pda_cache_desc* desc, const float* k_scale,
                                   const float* v_scale, const int32_t* block_table,

@@ -1,6 +1,7 @@
 // C ABI of libpda: argument validation on the host, then kernel dispatch.
 #include <atomic>
 #include <cstdint>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -91,6 +92,43 @@ int check_attention(const void* q, const void* k_cache, const void* v_cache,
 }  // namespace
 
 namespace {
+// A library-owned second stream for the one place where two independent launches of a call can share
+// the GPU (the shared-prefix cascade: its prefix launch leaves SMs idle that the suffix launch can use).
+// Fork and join go through events, so the pattern is also valid inside a stream capture. Created on the
+// first call that is not being captured (creating a stream during a capture is not allowed in every
+// capture mode); until then such calls run their launches one after the other. One process drives one
+// device here, so there is one of these.
+struct SideStream {
+  std::mutex mu;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+SideStream g_side;
+
+bool side_stream_ready(cudaStream_t main_stream) {  // g_side.mu held
+  if (g_side.stream) return true;
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(main_stream, &st) != cudaSuccess || st != cudaStreamCaptureStatusNone) {
+    cudaGetLastError();
+    return false;
+  }
+  cudaStream_t ns = nullptr;
+  cudaEvent_t a = nullptr, b = nullptr;
+  if (cudaStreamCreateWithFlags(&ns, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&b, cudaEventDisableTiming) != cudaSuccess) {
+    cudaGetLastError();
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (ns) cudaStreamDestroy(ns);
+    return false;
+  }
+  g_side.stream = ns;
+  g_side.fork = a;
+  g_side.join = b;
+  return true;
+}
+
 // Device address of pinned, mapped host memory (what cudaHostAlloc / cudaHostRegister give); NULL for
 // anything the device cannot reach.
 void* mapped_device_pointer(const void* host) {
@@ -295,6 +333,14 @@ int paged_prefix_decode_attention(const void* q, const void* k_cache, const void
   p.out = static_cast<__nv_bfloat16*>(out);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 
+  // The suffix launch (2) is independent of the prefix launch (1) and small, and (1) rarely fills the
+  // GPU (one CTA per SM, chunks x kv heads of them), so (2) runs beside it on the library's second
+  // stream: the fork event is recorded before (1), (1) is submitted first so that its CTAs are placed
+  // first, and (2) is joined before the merge.
+  std::lock_guard<std::mutex> lock(g_side.mu);
+  bool forked = side_stream_ready(s) && cudaEventRecord(g_side.fork, s) == cudaSuccess;
+  if (!forked) cudaGetLastError();
+
   // (1) the shared prefix once: the batch's queries as one block of rows per kv head
   AttnParams pp = p;
   pp.batch = 1;
@@ -312,7 +358,17 @@ int paged_prefix_decode_attention(const void* q, const void* k_cache, const void
   AttnParams ps = p;
   ps.first_token = prefix_tokens;
   ps.chunk_slot0 = prefix_chunks;
-  if (cudaError_t e = pda::launch_attention_tma(ps, s)) return static_cast<int>(e);
+  if (forked && cudaStreamWaitEvent(g_side.stream, g_side.fork, 0) != cudaSuccess) {
+    cudaGetLastError();
+    forked = false;
+  }
+  cudaError_t e2 = pda::launch_attention_tma(ps, forked ? g_side.stream : s);
+  if (forked) {  // join in any case: a capture must not be left with an open branch
+    cudaError_t ej = cudaEventRecord(g_side.join, g_side.stream);
+    if (ej == cudaSuccess) ej = cudaStreamWaitEvent(s, g_side.join, 0);
+    if (e2 == cudaSuccess) e2 = ej;
+  }
+  if (e2 != cudaSuccess) return static_cast<int>(e2);
   // (3) merge
   return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
                                              p.geom.head_dim, chunk_tokens, max_chunks,
