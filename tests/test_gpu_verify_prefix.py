@@ -117,3 +117,44 @@ def test_shared_prefix_cascade(oracle, kv_dtype, B, flags):
     plain = dw.attend()
     assert np.abs(bf16_to_f64(plain) - bf16_to_f64(out)).max() < 2e-2
     assert int(dw.status.item()) == 0
+
+
+def test_shared_prefix_cascade_in_a_cuda_graph(oracle):
+    """The cascade forks its suffix launch onto a library-owned stream; captured in a graph the fork
+    and join become graph edges. Replays must give the eager (and the oracle's) result."""
+    rng = np.random.default_rng(8)
+    prefix, B = 1024, 12
+    lens = prefix + rng.integers(1, 200, size=B)
+    w = W.make_workload("cascade_graph", lens, 32, 8, 128, seed=30, shared_prefix_tokens=prefix)
+    dw = DeviceWorkload(w)
+    dw.append()
+    from util import host_appended
+    k, v = host_appended(oracle, w)
+    ref = oracle_out(oracle, w, k, v)
+    pchunk, chunk = 256, 64
+    mc = prefix // pchunk + pda.max_chunks(int(lens.max()) - prefix + 1, chunk)
+    po = torch.empty((B, 32, mc, 128), dtype=torch.float32, device="cuda")
+    pl = torch.empty((B, 32, mc), dtype=torch.float32, device="cuda")
+    out = torch.empty_like(dw.q)
+
+    def run(stream=None):
+        pda.paged_prefix_decode_attention(dw.q, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                          float(w.scale), prefix, pchunk, chunk, po, pl, out=out,
+                                          status=dw.status, stream=stream)
+    run()                      # eager once: creates the side stream outside any capture
+    torch.cuda.synchronize()
+    eager = out.clone()
+    assert_close(bf16_to_f64(eager), ref, what="cascade eager")
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            run(s)
+    for _ in range(3):
+        out.zero_()
+        po.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), eager.view(torch.int16))
+    assert int(dw.status.item()) == 0
