@@ -83,7 +83,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.002)   # several samples even inside a timed region of a few ms
 
     def __enter__(self):
         if self.nv is not None:
