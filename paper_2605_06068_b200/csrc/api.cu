@@ -441,6 +441,8 @@ int paged_decode_reduce(const float* part_o, const float* part_lse, const int32_
   if (batch > 65535 || num_q_heads > 65535) return PDA_ERR_TOO_LARGE;
   if (batch == 0) return PDA_OK;
   if (!part_o || !part_lse || !seq_lens || !out) return PDA_ERR_INVALID_ARG;
+  if (head_dim % 4 != 0) return PDA_ERR_UNSUPPORTED;
+  if (!aligned16(part_o) || (reinterpret_cast<uintptr_t>(out) & 7u)) return PDA_ERR_MISALIGNED;
   return static_cast<int>(pda::launch_reduce(part_o, part_lse, seq_lens, batch, num_q_heads,
                                              head_dim, chunk_tokens, max_chunks, 0, 0, 1,
                                              static_cast<__nv_bfloat16*>(out),
