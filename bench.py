@@ -338,7 +338,7 @@ def run_gpu(args):
             pda.paged_decode_step_host(hq, hk, hv, hbt, hsl, st[0], st[1], st[2], dbt, dsl, k_cache, v_cache,
                                        float(w.scale), chunk, part_o, part_lse,
                                        None if in_place else out, out_host,
-                                       workspace=workspace if fused else None, status=status)
+                                       workspace=workspace if fused else None, status=status, stream=stream)
 
         def time_host(in_place):
             for _ in range(max(args.warmup, 3)):

@@ -460,6 +460,20 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
                            int32_t* status, pda_stream_t stream) {
   AttnParams p;
   if (!out_host || !q_host || !k_new_host || !v_new_host) return PDA_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The two copies every CTA depends on go first, so that they travel while the host is still busy
+  // with the rest of this call.
+  if (batch > 0 && block_table_host && seq_lens_host && block_table_dev && seq_lens_dev &&
+      block_table_stride > 0) {
+    cudaError_t e0;
+    if ((e0 = cudaMemcpyAsync(block_table_dev, block_table_host,
+                              static_cast<size_t>(batch) * block_table_stride * 4,
+                              cudaMemcpyHostToDevice, s)))
+      return e0;
+    if ((e0 = cudaMemcpyAsync(seq_lens_dev, seq_lens_host, static_cast<size_t>(batch) * 4,
+                              cudaMemcpyHostToDevice, s)))
+      return e0;
+  }
   // A staging buffer that is NULL means "in place": the kernel reads (writes) the host buffer itself
   // over the bus, which needs pinned, device-mapped host memory.
   const void* q_use = q_dev;
@@ -477,7 +491,6 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
   if (p.geom.dtype != PDA_BF16) return PDA_ERR_UNSUPPORTED;
   if (batch == 0) return PDA_OK;
   if (!block_table_host || !seq_lens_host) return PDA_ERR_INVALID_ARG;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t D = p.geom.head_dim;
   const size_t q_bytes = static_cast<size_t>(batch) * num_q_heads * D * 2;
   const size_t new_bytes = static_cast<size_t>(batch) * p.geom.num_kv_heads * D * 2;
@@ -485,13 +498,6 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
   if (q_dev && (e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, s))) return e;
   if (k_new_dev && (e = cudaMemcpyAsync(k_new_dev, k_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
   if (v_new_dev && (e = cudaMemcpyAsync(v_new_dev, v_new_host, new_bytes, cudaMemcpyHostToDevice, s))) return e;
-  if ((e = cudaMemcpyAsync(block_table_dev, block_table_host,
-                           static_cast<size_t>(batch) * block_table_stride * 4,
-                           cudaMemcpyHostToDevice, s)))
-    return e;
-  if ((e = cudaMemcpyAsync(seq_lens_dev, seq_lens_host, static_cast<size_t>(batch) * 4,
-                           cudaMemcpyHostToDevice, s)))
-    return e;
   if (int rc = paged_decode_step(q_use, k_use, v_use, k_cache, v_cache, desc, nullptr, nullptr,
                                  block_table_dev, block_table_stride, seq_lens_dev, batch,
                                  num_q_heads, scale, chunk_tokens, out_use, part_o, part_lse,
