@@ -424,6 +424,29 @@ def test_reduce_alone(oracle):
     assert torch.equal(out1.cpu(), expect)
 
 
+@pytest.mark.parametrize("D", [64, 128, 256])
+@pytest.mark.parametrize("Cm", [1, 33, 300])
+def test_reduce_many_chunks_and_widths(oracle, D, Cm):
+    """Chunk counts on both sides of the kernel's register-held weight blocks (32 per block, 256 in
+    registers, more recomputed), ragged per sequence, for every vector width of a row."""
+    rng = np.random.default_rng(Cm * 1000 + D)
+    B, Hq, chunk = 5, 3, 16
+    po = rng.standard_normal((B, Hq, Cm, D)).astype(np.float32)
+    pl = (rng.standard_normal((B, Hq, Cm)) * 4).astype(np.float32)
+    seq = np.array([Cm * chunk, max(Cm * chunk - 17, 1), (Cm // 2) * chunk + 1, 1, 0], np.int32)
+    for b in range(B):                      # chunks past a sequence's end hold poison and are never read
+        n = (int(seq[b]) + chunk - 1) // chunk
+        po[b, :, n:] = np.nan
+        pl[b, :, n:] = np.nan
+    pl[0, 1, 0] = -np.inf                   # an empty chunk inside the range: weight 0
+    po[0, 1, 0] = 0.0
+    ref, _ = oracle.paged_decode_reduce(po.astype(np.float64), pl.astype(np.float64), seq, chunk)
+    out = pda.paged_decode_reduce(torch.from_numpy(po).cuda(), torch.from_numpy(pl).cuda(),
+                                  torch.from_numpy(seq).cuda(), chunk)
+    assert_close(bf16_to_f64(out), ref, what=f"reduce Cm={Cm} D={D}", norm=False)
+    assert (bf16_to_f64(out)[4] == 0).all()
+
+
 # ---- the end-to-end host call ---------------------------------------------------------------
 
 def test_step_host_matches_device_calls(oracle):
