@@ -347,6 +347,28 @@ def test_fused_step_matches_oracle_and_appends_bit_exactly(oracle, case, step_ke
         assert np.abs(sep - bf16_to_f64(out)).max() <= 2.0 ** -7 * max(1e-30, np.abs(sep).max())
 
 
+@pytest.mark.parametrize("case", [([5000, 33, 700], 32, 8, 128, 16),      # 313 chunks: weights in shared memory
+                                  ([26000, 40], 8, 1, 64, 16)],             # 1625 chunks x 8 heads: do not fit, plain loop
+                         ids=["313chunks", "1625chunks"])
+def test_fused_step_merge_of_many_chunks(oracle, case):
+    lens, Hq, Hkv, D, chunk = case
+    w = W.make_workload("manychunks", lens, Hq, Hkv, D, seed=77)
+    k_ref, v_ref = host_appended(oracle, w)
+    ref = oracle_out(oracle, w, k_ref, v_ref)
+    dw = DeviceWorkload(w)
+    ws = pda.new_workspace(w.batch, Hkv)
+    mc = pda.max_chunks(max(lens), chunk)
+    po = torch.full((w.batch, Hq, mc, D), float("nan"), dtype=torch.float32, device="cuda")
+    pl = torch.full((w.batch, Hq, mc), float("nan"), dtype=torch.float32, device="cuda")
+    out = pda.paged_decode_step(dw.q, dw.k_new, dw.v_new, dw.k_cache, dw.v_cache, dw.block_table,
+                                dw.seq_lens, float(w.scale), chunk_tokens=chunk, part_o=po, part_lse=pl,
+                                workspace=ws, status=dw.status)
+    torch.cuda.synchronize()
+    assert_close(bf16_to_f64(out), ref, what=f"fused step, {mc} chunks")
+    assert (ws == 0).all() and status_of(dw) == 0
+    assert (bf16_to_bits(dw.k_cache) == k_ref).all()
+
+
 def test_fused_step_fp8_and_no_append(oracle):
     w = W.prefix_fp8(seed=46, batch=6)
     dw = DeviceWorkload(w)
