@@ -1,5 +1,5 @@
 // Multi-query paged attention on the 5th-generation tensor cores (tcgen05 + TMEM),
-// bf16 KV, head_dim 128. Same contract as attention_mq.cu (verification of a
+// bf16 KV, head_dim 128 or 64 (the figures in this comment are for 128). Same contract as attention_mq.cu (verification of a
 // block of draft tokens; the shared-prefix part of a decode batch): up to 128
 // query rows (query tokens x group size) per CTA against one sequence's pages.
 //
@@ -43,16 +43,20 @@ namespace pda {
 
 namespace {
 
-constexpr int kTcD = 128;               // head_dim
 constexpr int kTcRows = 128;            // query rows per CTA (UMMA M)
 constexpr int kTcPagesPerIter = 4;      // 64 tokens per iteration
-constexpr int kTcStages = 6;
-constexpr int kTcTileBytes = kPageSize * kTcD * 2;        // 4096: one K or V page tile
-constexpr int kTcKBytes = kTcPagesPerIter * kTcTileBytes;  // 16 KB: K of 4 pages as [2 lines][64 tokens][128 B]
-constexpr int kTcStageBytes = 2 * kTcKBytes;               // 32 KB: K block, then 4 V page tiles
 constexpr int kTcOnesBytes = 2048;                         // bf16 ones: B operand [16 tokens][16 columns] of the row-sum MMA
 constexpr int kTcMBytes = 2 * kTcRows * 4;                 // running row maxima handed between the two softmax sets
-constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + kTcOnesBytes + kTcMBytes + 256 + 1024;
+// Sizes that depend on head_dim D (128 or 64): a row is D / 64 lines of 128 bytes
+template <int D>
+struct TcCfg {
+  static constexpr int kLines = D / 64;
+  static constexpr int kTileBytes = kPageSize * D * 2;          // one K or V page tile: 4096 / 2048
+  static constexpr int kKBytes = kTcPagesPerIter * kTileBytes;  // K of 4 pages as [lines][64 tokens][128 B]
+  static constexpr int kStageBytes = 2 * kKBytes;               // K block, then 4 V page tiles: 32 / 16 KB
+  static constexpr int kStages = 6 * 128 / D;                   // 192 KB of ring either way
+  static constexpr int kSmemBytes = kStages * kStageBytes + kTcOnesBytes + kTcMBytes + 512 + 1024;
+};
 constexpr int kTcSoftmaxWarps = 8;      // two sets of 4: set x takes the iterations it with it % 2 == x
 constexpr int kTcProducerWarp = 8, kTcMmaWarp = 9, kTcPvWarp = 10;  // (the MMA warp issues S and owns the TMEM allocation)
 constexpr int kTcThreads = 352;
@@ -142,11 +146,14 @@ __device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
                        const __grid_constant__ CUtensorMap v_map, MqParams mp) {
   const AttnParams& p = mp.a;
-  constexpr int D = kTcD;
+  using C = TcCfg<D>;
+  constexpr int kTcStages = C::kStages, kTcStageBytes = C::kStageBytes, kTcKBytes = C::kKBytes,
+                kTcTileBytes = C::kTileBytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* ones_smem = smem + kTcStages * kTcStageBytes;
@@ -239,7 +246,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
     const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
+    for (int h = 0; h < D / 64; ++h) {  // 64 bf16 = 32 columns per store
       uint32_t qv[32];
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
@@ -280,8 +287,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         const int page_raw = __shfl_sync(0xffffffffu, pg, (it & 7) * kTcPagesPerIter + j);
         bad |= page_raw < 0;
         const int page = max(page_raw, 0);
-        tma_load_5d_if(leader, stage + j * (kPageSize * 128), &k_map, bar, 0, g, page);
-        tma_load_5d_if(leader, stage + kTcKBytes / 2 + j * (kPageSize * 128), &k_map, bar, 1, g, page);
+#pragma unroll
+        for (int ln = 0; ln < C::kLines; ++ln)
+          tma_load_5d_if(leader, stage + ln * (kTcKBytes / C::kLines) + j * (kPageSize * 128), &k_map, bar, ln, g, page);
         tma_load_5d_if(leader, stage + kTcKBytes + j * kTcTileBytes, &v_map, bar, 0, g, page);
       };
       if (n_here == kTcPagesPerIter) {
@@ -324,8 +332,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       const int tail = u_tail0 - (it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
       if (tail < kPageSize) {  // clear the rows past the sequence end in V (P is 0 there, V must be finite)
         const uint32_t vt = stage + kTcKBytes + (n_here - 1) * kTcTileBytes;
-        for (int i = lane; i < (kPageSize - tail) * 16; i += 32) {
-          const int r = tail + i / 16, ch = i % 16;
+        constexpr int kChunksPerRow = D / 8;  // 16-byte chunks of a row
+        for (int i = lane; i < (kPageSize - tail) * kChunksPerRow; i += 32) {
+          const int r = tail + i / kChunksPerRow, ch = i % kChunksPerRow;
           asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_off(r, ch)), "r"(0));
         }
         fence_proxy_async();
@@ -339,7 +348,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks) {
         // descriptor start addresses are in 16-byte units: +2 per k-step, next line block further on
-        const uint64_t bd = kd0 + static_cast<uint64_t>((ks >> 2) * (kTcKBytes / 2 / 16) + (ks & 3) * 2);
+        const uint64_t bd = kd0 + static_cast<uint64_t>((ks >> 2) * (kTcKBytes / C::kLines / 16) + (ks & 3) * 2);
         tc_mma_ts_if(leader, d, u_tmem + kTmemQ + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
       }
       tc_commit_if(leader, bar_s + 8 * (it & 1));
@@ -520,9 +529,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const float inv = live ? 1.f / l : 0.f;
     const int64_t qrow = (static_cast<int64_t>(b) * T + i_tok) * p.num_q_heads + g * G + (r % G);
     constexpr float kLn2 = 0.6931471805599453f;
-    // set x stores columns [64 x, 64 x + 64) of the row
+    // set x stores columns [D/2 x, D/2 (x + 1)) of the row, 32 at a time
 #pragma unroll
-    for (int cb = 2 * set; cb < 2 * set + 2; ++cb) {
+    for (int cb = (D / 64) * set; cb < (D / 64) * (set + 1); ++cb) {
       uint32_t ov[32];
       if (have) {
         tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
@@ -569,12 +578,28 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 
 bool attention_mq_tc_supports(const MqParams& mp) {
   const AttnParams& p = mp.a;
-  if (p.geom.dtype != PDA_BF16 || p.geom.head_dim != kTcD) return false;
+  if (p.geom.dtype != PDA_BF16 || (p.geom.head_dim != 128 && p.geom.head_dim != 64)) return false;
   if (p.group < 1 || mp.n_q < 1 || p.geom.num_pages < 1) return false;
   if (!(p.scale > 0.f) || !(p.scale < INFINITY)) return false;  // the row maximum is taken before scaling
   const int64_t rows = static_cast<int64_t>(mp.n_q) * p.group;
   return p.geom.num_kv_heads * ((rows + kTcRows - 1) / kTcRows) <= 65535;
 }
+
+namespace {
+template <int D>
+cudaError_t launch_tc(const CUtensorMap& k_map, const CUtensorMap& v_map, const MqParams& mp, cudaStream_t stream) {
+  const AttnParams& p = mp.a;
+  cudaError_t e = cudaFuncSetAttribute(attention_mq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       TcCfg<D>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  const int rows_total = mp.n_q * p.group;
+  const int n_rb = (rows_total + kTcRows - 1) / kTcRows;
+  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(mp.n_chunks_grid) : 1u;
+  dim3 grid(chunks, p.geom.num_kv_heads * n_rb, p.batch);
+  attention_mq_tc_kernel<D><<<grid, kTcThreads, TcCfg<D>::kSmemBytes, stream>>>(k_map, v_map, mp);
+  return cudaGetLastError();
+}
+}  // namespace
 
 cudaError_t launch_attention_mq_tc(const MqParams& mp, cudaStream_t stream) {
   const AttnParams& p = mp.a;
@@ -584,15 +609,7 @@ cudaError_t launch_attention_mq_tc(const MqParams& mp, cudaStream_t stream) {
       !make_cache_tensor_map(&v_map, p.v_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
                              p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2))
     return cudaErrorNotSupported;
-  cudaError_t e = cudaFuncSetAttribute(attention_mq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kTcSmemBytes);
-  if (e != cudaSuccess) return e;
-  const int rows_total = mp.n_q * p.group;
-  const int n_rb = (rows_total + kTcRows - 1) / kTcRows;
-  const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(mp.n_chunks_grid) : 1u;
-  dim3 grid(chunks, p.geom.num_kv_heads * n_rb, p.batch);
-  attention_mq_tc_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(k_map, v_map, mp);
-  return cudaGetLastError();
+  return p.geom.head_dim == 128 ? launch_tc<128>(k_map, v_map, mp, stream) : launch_tc<64>(k_map, v_map, mp, stream);
 }
 
 }  // namespace pda
