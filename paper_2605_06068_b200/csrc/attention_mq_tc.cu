@@ -1,5 +1,10 @@
 // Multi-query paged attention on the 5th-generation tensor cores (tcgen05 + TMEM),
-// bf16 KV, head_dim 128 or 64 (the figures in this comment are for 128). Same contract as attention_mq.cu (verification of a
+// bf16 KV with head_dim 128 or 64 (the figures in this comment are for 128), or e4m3 KV with head_dim
+// 128. The tensor core has no bf16 x e4m3 mode and e4m3 x e4m3 would quantise Q and P, so e4m3 tiles are
+// converted: the TMA ring holds the raw tiles, four converter warps write them as f16 operand blocks
+// (exact conversion, the page's scale folded in, rows past the sequence end zeroed) into three
+// conversion slots, and Q, P and the tile of ones are f16 as well. That variant runs 16 warps as four
+// warpgroups and redistributes registers between them (setmaxnreg). Same contract as attention_mq.cu (verification of a
 // block of draft tokens; the shared-prefix part of a decode batch): up to 128
 // query rows (query tokens x group size) per CTA against one sequence's pages.
 //
@@ -47,19 +52,33 @@ constexpr int kTcRows = 128;            // query rows per CTA (UMMA M)
 constexpr int kTcPagesPerIter = 4;      // 64 tokens per iteration
 constexpr int kTcOnesBytes = 2048;                         // bf16 ones: B operand [16 tokens][16 columns] of the row-sum MMA
 constexpr int kTcMBytes = 2 * kTcRows * 4;                 // running row maxima handed between the two softmax sets
-// Sizes that depend on head_dim D (128 or 64): a row is D / 64 lines of 128 bytes
-template <int D>
+// Sizes that depend on head_dim D (128 or 64) and on the cache's element type. A 16-bit row is D / 64
+// lines of 128 bytes. An operand block = what the tensor core reads for one iteration: K of 4 pages as
+// [lines][64 tokens][128 B], then 4 V page tiles. bf16 caches: the TMA ring holds operand blocks. e4m3
+// caches (D = 128): the ring holds the raw tiles (128-byte rows) and four converter warps turn them into
+// f16 operand blocks, exactly and with the page's scales folded in, in kConvSlots conversion slots.
+template <int D, bool kFp8>
 struct TcCfg {
+  static_assert(!kFp8 || D == 128, "e4m3 is built for head_dim 128");
   static constexpr int kLines = D / 64;
-  static constexpr int kTileBytes = kPageSize * D * 2;          // one K or V page tile: 4096 / 2048
+  static constexpr int kTileBytes = kPageSize * D * 2;          // one 16-bit K or V page tile: 4096 / 2048
   static constexpr int kKBytes = kTcPagesPerIter * kTileBytes;  // K of 4 pages as [lines][64 tokens][128 B]
-  static constexpr int kStageBytes = 2 * kKBytes;               // K block, then 4 V page tiles: 32 / 16 KB
-  static constexpr int kStages = 6 * 128 / D;                   // 192 KB of ring either way
-  static constexpr int kSmemBytes = kStages * kStageBytes + kTcOnesBytes + kTcMBytes + 512 + 1024;
+  static constexpr int kOperandBytes = 2 * kKBytes;             // K block, then 4 V page tiles: 32 / 16 KB
+  static constexpr int kRawTileBytes = kPageSize * D;           // one e4m3 page tile: 2048
+  static constexpr int kStageBytes = kFp8 ? 2 * kTcPagesPerIter * kRawTileBytes : kOperandBytes;
+  static constexpr int kStages = kFp8 ? 6 : 6 * 128 / D;        // 192 KB of ring for 16-bit caches, 96 KB for e4m3
+  static constexpr int kConvSlots = kFp8 ? 3 : 0;
+  static constexpr int kScaleBytes = kFp8 ? kStages * 2 * kTcPagesPerIter * 4 : 0;  // per stage: 4 K and 4 V scales
+  static constexpr int kSmemBytes = kStages * kStageBytes + kConvSlots * kOperandBytes + kTcOnesBytes + kTcMBytes +
+                                    kScaleBytes + 512 + 1024;
+  // warps: softmax 0-7; then (e4m3: converters 8-11) producer, S issue (+ TMEM allocation), PV issue
+  static constexpr int kProducerWarp = kFp8 ? 12 : 8, kMmaWarp = kProducerWarp + 1, kPvWarp = kProducerWarp + 2;
+  static constexpr int kThreads = kFp8 ? 512 : 352;
 };
 constexpr int kTcSoftmaxWarps = 8;      // two sets of 4: set x takes the iterations it with it % 2 == x
-constexpr int kTcProducerWarp = 8, kTcMmaWarp = 9, kTcPvWarp = 10;  // (the MMA warp issues S and owns the TMEM allocation)
-constexpr int kTcThreads = 352;
+// e4m3 variant: four warpgroups whose registers are redistributed at the start (setmaxnreg):
+// 2 x 128 x 176 (softmax) + 128 x 80 (converters) + 128 x 64 (producer, issuers, one spare warp) <= 65536
+constexpr uint32_t kTcRegsSoftmax = 176, kTcRegsConvert = 80, kTcRegsControl = 64;
 // Tensor memory columns (32-bit each, 128 lanes = query rows): S buffers 0..63 and 64..127 (f32),
 // O 128..255 (f32), Q 256..319 (bf16 pairs along d), P buffers 320..351 and 352..383 (bf16 pairs
 // along tokens). Allocations are powers of two.
@@ -101,10 +120,24 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lbo_byt
          (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) |
          (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: f32 accumulate, bf16 A and B, A K-major, M = 128.
-__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+// Instruction descriptor: f32 accumulate, A and B both bf16 or both f16, A K-major, M = 128.
+__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major, bool f16) {
+  return (1u << 4) | ((f16 ? 0u : 1u) << 7) | ((f16 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) |
          (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTcRows >> 4) << 24);
+}
+template <uint32_t kRegs>
+__device__ __forceinline__ void reg_alloc_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs)); }
+template <uint32_t kRegs>
+__device__ __forceinline__ void reg_alloc_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs)); }
+// 16 e4m3 values (one 16-byte chunk) -> 16 f16 values times a scale, as two 16-byte chunks
+__device__ __forceinline__ void e4m3x16_to_f16(const uint4& in, uint32_t scale2, uint4& lo, uint4& hi) {
+  auto cv = [&](uint32_t w, uint32_t& a, uint32_t& b) {
+    a = e4m3x2_to_f16x2(w & 0xffffu);
+    b = e4m3x2_to_f16x2(w >> 16);
+    asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(a) : "r"(scale2));
+    asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b) : "r"(scale2));
+  };
+  cv(in.x, lo.x, lo.y); cv(in.y, lo.z, lo.w); cv(in.z, hi.x, hi.y); cv(in.w, hi.z, hi.w);
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -146,21 +179,24 @@ __device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-template <int D>
-__global__ void __launch_bounds__(kTcThreads, 1)
+template <int D, bool kFp8>
+__global__ void __launch_bounds__((TcCfg<D, kFp8>::kThreads), 1)
 attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
                        const __grid_constant__ CUtensorMap v_map, MqParams mp) {
   const AttnParams& p = mp.a;
-  using C = TcCfg<D>;
+  using C = TcCfg<D, kFp8>;
   constexpr int kTcStages = C::kStages, kTcStageBytes = C::kStageBytes, kTcKBytes = C::kKBytes,
-                kTcTileBytes = C::kTileBytes;
+                kTcTileBytes = C::kTileBytes, kTcThreads = C::kThreads;
+  constexpr int kTcProducerWarp = C::kProducerWarp, kTcMmaWarp = C::kMmaWarp, kTcPvWarp = C::kPvWarp;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* ones_smem = smem + kTcStages * kTcStageBytes;
+  uint8_t* conv_smem = smem + kTcStages * kTcStageBytes;             // e4m3: kConvSlots operand blocks
+  uint8_t* ones_smem = conv_smem + C::kConvSlots * C::kOperandBytes;
   float* m_sh = reinterpret_cast<float*>(ones_smem + kTcOnesBytes);        // [2][128]
-  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 10);
+  float* scale_sh = m_sh + 2 * kTcRows;                                    // e4m3: [stage][4 K scales, 4 V scales]
+  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2], conv_full[3], conv_free[3]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes + C::kScaleBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 16);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -208,12 +244,18 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
   const uint32_t bar_sfree = bar_pv + 16, bar_m = bar_sfree + 16;
-  for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads) reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;
+  const uint32_t conv_full0 = bar_m + 16, conv_free0 = conv_full0 + 24;  // three of each (e4m3)
+  for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads)
+    reinterpret_cast<uint32_t*>(ones_smem)[i] = kFp8 ? 0x3C003C00u : 0x3F803F80u;  // 1.0 as f16 / bf16 pairs
   fence_proxy_async();  // read by the tensor core through the async proxy
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full0 + 8 * s, 1);
-      mbar_init(empty0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, kFp8 ? 4 : 1);  // released by the PV MMAs' commit, or by the 4 converter warps
+    }
+    for (int k = 0; k < 3; ++k) {
+      mbar_init(conv_full0 + 8 * k, 4);  // an operand block converted (4 converter warps)
+      mbar_init(conv_free0 + 8 * k, 1);  // the PV MMAs that read it have completed
     }
     for (int k = 0; k < 2; ++k) {
       mbar_init(bar_s + 8 * k, 1);
@@ -239,33 +281,51 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTmemO;  // S buffer k at tmem_s + 64 k
   const uint32_t tmem_q = tmem_base + kTmemQ, tmem_p = tmem_base + kTmemP;  // P buffer k at tmem_p + 32 k
 
-  // ---- Q: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of S = Q . K^T
-  if (warp < 4) {
-    const int r = rb * kTcRows + tid;
-    const bool valid = r < rows_total;
-    const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
-    const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
-#pragma unroll
-    for (int h = 0; h < D / 64; ++h) {  // 64 bf16 = 32 columns per store
-      uint32_t qv[32];
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const uint4 v = valid ? src[h * 8 + ch] : make_uint4(0u, 0u, 0u, 0u);
-        qv[4 * ch] = v.x; qv[4 * ch + 1] = v.y; qv[4 * ch + 2] = v.z; qv[4 * ch + 3] = v.w;
-      }
-      tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32 * h, qv);
-    }
-    tmem_wait_st();
-  }
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
 
-  if (warp == kTcProducerWarp) {
+  // The roles, as closures: the two variants dispatch them differently (the e4m3 one by warpgroup, each
+  // group first taking or giving up registers).
+  // ---- Q: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of S = Q . K^T
+  auto load_q = [&]() {
+    if (warp < 4) {
+      const int r = rb * kTcRows + tid;
+      const bool valid = r < rows_total;
+      const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
+  #pragma unroll
+      for (int h = 0; h < D / 64; ++h) {  // 64 bf16 = 32 columns per store
+        uint32_t qv[32];
+  #pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint4 v = valid ? src[h * 8 + ch] : make_uint4(0u, 0u, 0u, 0u);
+          qv[4 * ch] = v.x; qv[4 * ch + 1] = v.y; qv[4 * ch + 2] = v.z; qv[4 * ch + 3] = v.w;
+          if (kFp8) {  // the e4m3 variant multiplies in f16: bf16 pairs -> f16 pairs
+  #pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const uint32_t w = qv[4 * ch + e];
+              qv[4 * ch + e] = pack2<true>(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+            }
+          }
+        }
+        tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32 * h, qv);
+      }
+      tmem_wait_st();
+    }
+  };
+  auto wait_q = [&]() {
+    // Q is in tensor memory before the first MMA is issued (the producer does not take part)
+    tc_fence_before();
+    asm volatile("bar.sync 1, %0;" ::"n"(kTcThreads - 32) : "memory");
+    tc_fence_after();
+  };
+  auto producer_role = [&]() {
     // ================= TMA producer (does not wait for Q) =================
     const uint32_t leader = elect_one();
     const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     bool bad = false;
     int pg = 0;
+    float ks = 0.f, vs = 0.f;  // e4m3: the page's dequantisation factors
     for (int it = 0; it < u_iters; ++it) {
       const int s = it % kTcStages;
       if ((it & 7) == 0) {  // page ids of the next 8 iterations (32 pages), one per lane
@@ -273,6 +333,10 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         if (it * kTcPagesPerIter + lane < u_pages) {
           const int v = table[page0 + it * kTcPagesPerIter + lane];
           pg = (v < 0 || v >= p.geom.num_pages) ? -1 : v;
+          if (kFp8) {
+            ks = p.k_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g];
+            vs = p.v_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g];
+          }
         }
       }
       bool ok = true;
@@ -281,16 +345,29 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       const uint32_t stage = ring + s * kTcStageBytes, bar = full0 + 8 * s;
-      mbar_expect_tx_if(leader, bar, n_here * 2 * kTcTileBytes);
+      if (kFp8) {  // this stage's scales, written by the lanes that hold its pages (seen through the full barrier)
+        if ((lane >> 2) == (it & 7)) {
+          scale_sh[s * 8 + (lane & 3)] = ks;
+          scale_sh[s * 8 + 4 + (lane & 3)] = vs;
+        }
+        __syncwarp();
+      }
+      mbar_expect_tx_if(leader, bar, n_here * 2 * (kFp8 ? C::kRawTileBytes : kTcTileBytes));
       // K: one copy per 128-byte line so that page j's 16 rows follow page j-1's in each line block
+      // (an e4m3 row is one line; raw V tiles follow the raw K block)
       auto load_page = [&](int j) {
         const int page_raw = __shfl_sync(0xffffffffu, pg, (it & 7) * kTcPagesPerIter + j);
         bad |= page_raw < 0;
         const int page = max(page_raw, 0);
+        if (kFp8) {
+          tma_load_5d_if(leader, stage + j * C::kRawTileBytes, &k_map, bar, 0, g, page);
+          tma_load_5d_if(leader, stage + (kTcPagesPerIter + j) * C::kRawTileBytes, &v_map, bar, 0, g, page);
+        } else {
 #pragma unroll
-        for (int ln = 0; ln < C::kLines; ++ln)
-          tma_load_5d_if(leader, stage + ln * (kTcKBytes / C::kLines) + j * (kPageSize * 128), &k_map, bar, ln, g, page);
-        tma_load_5d_if(leader, stage + kTcKBytes + j * kTcTileBytes, &v_map, bar, 0, g, page);
+          for (int ln = 0; ln < C::kLines; ++ln)
+            tma_load_5d_if(leader, stage + ln * (kTcKBytes / C::kLines) + j * (kPageSize * 128), &k_map, bar, ln, g, page);
+          tma_load_5d_if(leader, stage + kTcKBytes + j * kTcTileBytes, &v_map, bar, 0, g, page);
+        }
       };
       if (n_here == kTcPagesPerIter) {
 #pragma unroll
@@ -300,19 +377,14 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
     }
     if (bad && lane == 0) atomicMax(cta_err, PDA_DEV_BAD_PAGE);
-  } else {
-    // Q is in tensor memory before the first MMA is issued (the producer does not take part)
-    tc_fence_before();
-    asm volatile("bar.sync 1, %0;" ::"n"(kTcThreads - 32) : "memory");
-    tc_fence_after();
-  }
-  if (warp == kTcMmaWarp) {
+  };
+  auto s_issue_role = [&]() {
     // ================= S issue: S(it) = Q . K^T as soon as its operands allow =================
     // (Two issuing warps, one for S and one for PV: a single warp runs the few hundred dependent scalar
     // instructions of both per iteration at one every 4-8 clocks, which is as long as the iteration
     // itself. Each keeps to its own chain of barriers; the tensor core's order between the two does not
     // matter.)
-    constexpr uint32_t idesc_s = tc_idesc(kTcPagesPerIter * kPageSize, false);
+    constexpr uint32_t idesc_s = tc_idesc(kTcPagesPerIter * kPageSize, false, kFp8);
     const uint32_t leader = elect_one();
     // warp-uniform copies (a shuffle from lane 0 tells the compiler so)
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
@@ -320,17 +392,23 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     const int u_tail0 = __shfl_sync(0xffffffffu, L - page0 * kPageSize, 0);  // tokens from the first page to the end
     bool ok = true;
-    uint32_t stage_i = 0, stage_par = 0;  // the iteration's ring stage and that stage's phase parity
+    // the iteration's operand block: its ring stage (16-bit caches) or conversion slot (e4m3), and the
+    // phase parity of that block's "ready" barrier
+    constexpr uint32_t kBlocks = kFp8 ? C::kConvSlots : kTcStages;
+    const uint32_t blocks0 = kFp8 ? smem_u32(conv_smem) : ring;
+    const uint32_t ready0 = kFp8 ? conv_full0 : full0;
+    uint32_t stage_i = 0, stage_par = 0;
     for (int it = 0; it < u_iters; ++it) {
       // S(it) overwrites the buffer of S(it-2): the softmax warps have loaded that into registers
       if (it >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (it & 1), ((it - 2) >> 1) & 1);
-      if (ok) ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);  // the stage has landed
+      if (ok) ok = mbar_wait_bounded(ready0 + 8 * stage_i, stage_par);  // the block has landed / been converted
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      const uint32_t stage = ring + stage_i * kTcStageBytes;
+      const uint32_t stage = blocks0 + stage_i * C::kOperandBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       const int tail = u_tail0 - (it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
-      if (tail < kPageSize) {  // clear the rows past the sequence end in V (P is 0 there, V must be finite)
+      if (!kFp8 && tail < kPageSize) {  // clear the rows past the sequence end in V (P is 0 there, V must be
+                                        // finite); the e4m3 converters do it as they write the block
         const uint32_t vt = stage + kTcKBytes + (n_here - 1) * kTcTileBytes;
         constexpr int kChunksPerRow = D / 8;  // 16-byte chunks of a row
         for (int i = lane; i < (kPageSize - tail) * kChunksPerRow; i += 32) {
@@ -352,26 +430,29 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         tc_mma_ts_if(leader, d, u_tmem + kTmemQ + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
       }
       tc_commit_if(leader, bar_s + 8 * (it & 1));
-      if (++stage_i == kTcStages) { stage_i = 0; stage_par ^= 1; }
+      if (++stage_i == kBlocks) { stage_i = 0; stage_par ^= 1; }
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
-  } else if (warp == kTcPvWarp) {
+  };
+  auto pv_issue_role = [&]() {
     // ================= PV issue: O += P . V and l += P . 1 =================
-    constexpr uint32_t idesc_pv = tc_idesc(D, true);
-    constexpr uint32_t idesc_l = tc_idesc(16, false);
+    constexpr uint32_t idesc_pv = tc_idesc(D, true, kFp8);
+    constexpr uint32_t idesc_l = tc_idesc(16, false, kFp8);
     const uint64_t ones_desc = tc_desc(smem_u32(ones_smem), 16, 1024);
     const uint32_t leader = elect_one();
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
     const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     bool ok = true;
-    uint32_t stage_i = 0;
+    constexpr uint32_t kBlocks = kFp8 ? C::kConvSlots : kTcStages;
+    const uint32_t blocks0 = kFp8 ? smem_u32(conv_smem) : ring;
+    uint32_t stage_i = 0;  // the iteration's operand block: ring stage or conversion slot
     for (int it = 0; it < u_iters; ++it) {
       ok = mbar_wait_bounded(bar_p + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t stage = ring + stage_i * kTcStageBytes;
+      const uint32_t stage = blocks0 + stage_i * C::kOperandBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page, V read MN-major
       const uint32_t pa0 = u_tmem + kTmemP + 32 * (it & 1);
@@ -388,12 +469,75 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       } else {
         for (int j = 0; j < n_here; ++j) pv_page(j);
       }
-      tc_commit_if(leader, empty0 + 8 * stage_i);     // the stage may be refilled once these MMAs have read it
+      // the stage may be refilled (the conversion slot rewritten) once these MMAs have read it
+      tc_commit_if(leader, (kFp8 ? conv_free0 : empty0) + 8 * stage_i);
       tc_commit_if(leader, bar_pv + 8 * (it & 1));    // O and l updated, P buffer free again
-      if (++stage_i == kTcStages) stage_i = 0;
+      if (++stage_i == kBlocks) stage_i = 0;
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
-  } else if (warp < kTcSoftmaxWarps) {
+  };
+  auto convert_role = [&]() {
+    if constexpr (kFp8) {
+      // ================= e4m3 -> f16 converters: raw stage -> operand block in a conversion slot ==========
+      // cvt.rn.f16x2.e4m3x2 is exact, the page's scale is folded in (one f16 multiply), rows past the
+      // sequence end become zeros. A thread moves 4 K and 4 V chunks of 16 bytes per iteration: raw row r,
+      // chunk c (swizzled by the row) -> 16-bit row r, chunks 2 (c % 4), 2 (c % 4) + 1 of line c / 4.
+      const int ct = tid - kTcSoftmaxWarps * 32;  // 0..127
+      const uint32_t conv0 = smem_u32(conv_smem);
+      uint32_t slot = 0, slot_par = 0, stage_i = 0, stage_par = 0;
+      bool ok = true;
+      for (int it = 0; it < n_iters; ++it) {
+        ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);                        // raw tiles have landed
+        if (ok && it >= C::kConvSlots) ok = mbar_wait_bounded(conv_free0 + 8 * slot, slot_par ^ 1);  // PV(it - 3) done
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t raw = ring + stage_i * kTcStageBytes;
+        const uint32_t dst = conv0 + slot * C::kOperandBytes;
+        const float* sc = scale_sh + stage_i * 8;
+        const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
+        const int valid_rows = min(L - (page0 + it * kTcPagesPerIter) * kPageSize, n_here * kPageSize);  // token rows of this block
+  #pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const int idx = q4 * 128 + ct;            // chunk index: 64 rows x 8 chunks
+          const int r = idx >> 3, c = idx & 7;      // stacked token row (page r / 16, slot r % 16), raw chunk
+          const int pj = r >> 4, rr = r & 15;
+          if (pj < n_here) {
+            const uint32_t src_off = static_cast<uint32_t>(pj * C::kRawTileBytes + rr * 128 + ((c ^ (rr & 7)) << 4));
+            const int line = c >> 2, c2 = (c & 3) * 2;
+            // K: [line][64 rows][128 B], row r; V: page tile pj = [line][16 rows][128 B], row rr
+            const uint32_t k_dst = dst + line * (64 * 128) + r * 128;
+            const uint32_t v_dst = dst + kTcKBytes + pj * kTcTileBytes + line * (kPageSize * 128) + rr * 128;
+            const int sw = r & 7;  // (== rr & 7)
+            uint4 kin, vin, lo, hi;
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kin.x), "=r"(kin.y), "=r"(kin.z), "=r"(kin.w) : "r"(raw + src_off));
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(vin.x), "=r"(vin.y), "=r"(vin.z), "=r"(vin.w)
+                         : "r"(raw + kTcPagesPerIter * C::kRawTileBytes + src_off));
+            const bool live = r < valid_rows;
+            const uint32_t ks2 = pack2<true>(sc[pj], sc[pj]);
+            const uint32_t vs2 = pack2<true>(sc[4 + pj], sc[4 + pj]);
+            e4m3x16_to_f16(kin, ks2, lo, hi);
+            if (!live) { lo = make_uint4(0u, 0u, 0u, 0u); hi = lo; }
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(k_dst + ((c2 ^ sw) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w));
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(k_dst + (((c2 + 1) ^ sw) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w));
+            e4m3x16_to_f16(vin, vs2, lo, hi);
+            if (!live) { lo = make_uint4(0u, 0u, 0u, 0u); hi = lo; }
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(v_dst + ((c2 ^ sw) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w));
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(v_dst + (((c2 + 1) ^ sw) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w));
+          }
+        }
+        fence_proxy_async();   // the tensor core reads the block through the async proxy
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_tc(conv_full0 + 8 * slot);   // block ready for S and PV
+          mbar_arrive_tc(empty0 + 8 * stage_i);    // raw stage may be refilled
+        }
+        if (++slot == C::kConvSlots) { slot = 0; slot_par ^= 1; }
+        if (++stage_i == kTcStages) { stage_i = 0; stage_par ^= 1; }
+      }
+      if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
+    }
+  };
+  auto softmax_role = [&]() {
     // ================= softmax: TMEM lane t <-> query row t; set x takes iterations x, x+2, ... ==========
     // Two warps per scheduler, one of each set: while one waits (for S, for the other set's row maximum,
     // for its tcgen05.ld/st) the other keeps the exp2 unit busy, which is what bounds this part.
@@ -487,7 +631,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         const uint64_t x2 = fma_f32x2(f32x2(sv[j >> 4][(2 * j) & 31], sv[j >> 4][(2 * j + 1) & 31]), c2, nr2);
         float x0, x1;
         f32x2_split(x2, x0, x1);
-        pw[j] = pack2<false>(ex2(x0), ex2(x1));
+        pw[j] = pack2<kFp8>(ex2(x0), ex2(x1));  // (f16 pairs in the e4m3 variant, bf16 otherwise)
       }
       tmem_st32(tmem_p + 32 * set + lane_base, pw);
       tmem_wait_st();
@@ -563,7 +707,37 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     }
     if (split && valid_row && set == 0)
       p.part_lse[qrow * p.max_chunks + p.chunk_slot0 + c] = live ? (m_ref + __log2f(l)) * kLn2 : -INFINITY;
+  };
+  if constexpr (!kFp8) {
+    load_q();
+    if (warp == kTcProducerWarp) producer_role(); else wait_q();
+    if (warp == kTcMmaWarp) s_issue_role();
+    else if (warp == kTcPvWarp) pv_issue_role();
+    else if (warp < kTcSoftmaxWarps) softmax_role();
+  } else {
+    // four warpgroups; registers go from the converter and control warps to the softmax warps (each group
+    // executes its setmaxnreg at the head of the code that only it runs)
+    if (warp < kTcSoftmaxWarps) {
+      reg_alloc_inc<kTcRegsSoftmax>();
+      load_q();
+      wait_q();
+      softmax_role();
+    } else if (warp < kTcSoftmaxWarps + 4) {
+      reg_alloc_dec<kTcRegsConvert>();
+      wait_q();
+      convert_role();
+    } else {
+      reg_alloc_dec<kTcRegsControl>();
+      if (warp == kTcProducerWarp) {
+        producer_role();
+      } else {
+        wait_q();
+        if (warp == kTcMmaWarp) s_issue_role();
+        else if (warp == kTcPvWarp) pv_issue_role();
+      }
+    }
   }
+
 
   // ---- teardown: everyone is done with tensor memory before it is released
   tc_fence_before();
@@ -578,7 +752,11 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 
 bool attention_mq_tc_supports(const MqParams& mp) {
   const AttnParams& p = mp.a;
-  if (p.geom.dtype != PDA_BF16 || (p.geom.head_dim != 128 && p.geom.head_dim != 64)) return false;
+  if (p.geom.dtype == PDA_BF16) {
+    if (p.geom.head_dim != 128 && p.geom.head_dim != 64) return false;
+  } else {
+    if (p.geom.head_dim != 128 || p.k_scale == nullptr || p.v_scale == nullptr) return false;
+  }
   if (p.group < 1 || mp.n_q < 1 || p.geom.num_pages < 1) return false;
   if (!(p.scale > 0.f) || !(p.scale < INFINITY)) return false;  // the row maximum is taken before scaling
   const int64_t rows = static_cast<int64_t>(mp.n_q) * p.group;
@@ -586,30 +764,36 @@ bool attention_mq_tc_supports(const MqParams& mp) {
 }
 
 namespace {
-template <int D>
+template <int D, bool kFp8>
 cudaError_t launch_tc(const CUtensorMap& k_map, const CUtensorMap& v_map, const MqParams& mp, cudaStream_t stream) {
   const AttnParams& p = mp.a;
-  cudaError_t e = cudaFuncSetAttribute(attention_mq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       TcCfg<D>::kSmemBytes);
+  using C = TcCfg<D, kFp8>;
+  cudaError_t e = cudaFuncSetAttribute(attention_mq_tc_kernel<D, kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       C::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int rows_total = mp.n_q * p.group;
   const int n_rb = (rows_total + kTcRows - 1) / kTcRows;
   const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(mp.n_chunks_grid) : 1u;
   dim3 grid(chunks, p.geom.num_kv_heads * n_rb, p.batch);
-  attention_mq_tc_kernel<D><<<grid, kTcThreads, TcCfg<D>::kSmemBytes, stream>>>(k_map, v_map, mp);
+  attention_mq_tc_kernel<D, kFp8><<<grid, C::kThreads, C::kSmemBytes, stream>>>(k_map, v_map, mp);
   return cudaGetLastError();
 }
 }  // namespace
 
 cudaError_t launch_attention_mq_tc(const MqParams& mp, cudaStream_t stream) {
   const AttnParams& p = mp.a;
+  const bool fp8 = p.geom.dtype != PDA_BF16;
+  const int eb = fp8 ? 1 : 2;
   alignas(64) CUtensorMap k_map, v_map;
+  // K is copied one 128-byte line of its rows at a time (so that the pages of an iteration stack), V as whole tiles
   if (!make_cache_tensor_map(&k_map, p.k_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
-                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2, /*box_lines=*/1) ||
+                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, eb, /*box_lines=*/1) ||
       !make_cache_tensor_map(&v_map, p.v_cache, p.geom.page_stride, p.geom.head_stride, p.geom.slot_stride,
-                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, 2))
+                             p.geom.num_pages, p.geom.num_kv_heads, p.geom.head_dim, eb))
     return cudaErrorNotSupported;
-  return p.geom.head_dim == 128 ? launch_tc<128>(k_map, v_map, mp, stream) : launch_tc<64>(k_map, v_map, mp, stream);
+  if (fp8) return launch_tc<128, true>(k_map, v_map, mp, stream);
+  return p.geom.head_dim == 128 ? launch_tc<128, false>(k_map, v_map, mp, stream)
+                                : launch_tc<64, false>(k_map, v_map, mp, stream);
 }
 
 }  // namespace pda
