@@ -67,6 +67,9 @@ struct TcCfg {
   static constexpr int kRawTileBytes = kPageSize * D;           // one e4m3 page tile: 2048
   static constexpr int kStageBytes = kFp8 ? 2 * kTcPagesPerIter * kRawTileBytes : kOperandBytes;
   static constexpr int kStages = kFp8 ? 6 : 6 * 128 / D;        // 192 KB of ring for 16-bit caches, 96 KB for e4m3
+  // (a slot is free again after the PV that read it; four slots with four raw stages, and separate pools
+  // for K and V, were measured no faster: the converters' instructions share the schedulers with the
+  // softmax warps, which is what stretches an iteration from 0.72 to 1.0 us)
   static constexpr int kConvSlots = kFp8 ? 3 : 0;
   static constexpr int kScaleBytes = kFp8 ? kStages * 2 * kTcPagesPerIter * 4 : 0;  // per stage: 4 K and 4 V scales
   static constexpr int kSmemBytes = kStages * kStageBytes + kConvSlots * kOperandBytes + kTcOnesBytes + kTcMBytes +
@@ -194,9 +197,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   uint8_t* ones_smem = conv_smem + C::kConvSlots * C::kOperandBytes;
   float* m_sh = reinterpret_cast<float*>(ones_smem + kTcOnesBytes);        // [2][128]
   float* scale_sh = m_sh + 2 * kTcRows;                                    // e4m3: [stage][4 K scales, 4 V scales]
-  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2], conv_full[3], conv_free[3]
+  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2], conv_full[4], conv_free[4]
   uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes + C::kScaleBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 16);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 18);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -244,7 +247,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
   const uint32_t bar_sfree = bar_pv + 16, bar_m = bar_sfree + 16;
-  const uint32_t conv_full0 = bar_m + 16, conv_free0 = conv_full0 + 24;  // three of each (e4m3)
+  const uint32_t conv_full0 = bar_m + 16, conv_free0 = conv_full0 + 32;  // four of each (e4m3)
   for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads)
     reinterpret_cast<uint32_t*>(ones_smem)[i] = kFp8 ? 0x3C003C00u : 0x3F803F80u;  // 1.0 as f16 / bf16 pairs
   fence_proxy_async();  // read by the tensor core through the async proxy
@@ -253,7 +256,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, kFp8 ? 4 : 1);  // released by the PV MMAs' commit, or by the 4 converter warps
     }
-    for (int k = 0; k < 3; ++k) {
+    for (int k = 0; k < 4; ++k) {
       mbar_init(conv_full0 + 8 * k, 4);  // an operand block converted (4 converter warps)
       mbar_init(conv_free0 + 8 * k, 1);  // the PV MMAs that read it have completed
     }
@@ -480,15 +483,24 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     if constexpr (kFp8) {
       // ================= e4m3 -> f16 converters: raw stage -> operand block in a conversion slot ==========
       // cvt.rn.f16x2.e4m3x2 is exact, the page's scale is folded in (one f16 multiply), rows past the
-      // sequence end become zeros. A thread moves 4 K and 4 V chunks of 16 bytes per iteration: raw row r,
-      // chunk c (swizzled by the row) -> 16-bit row r, chunks 2 (c % 4), 2 (c % 4) + 1 of line c / 4.
+      // sequence end become zeros. A thread moves 4 K and 4 V chunks of 16 bytes per iteration (one of each
+      // per page): raw row, chunk c (swizzled by the row) -> 16-bit row, chunks 2 (c % 4), 2 (c % 4) + 1 of
+      // line c / 4.
       const int ct = tid - kTcSoftmaxWarps * 32;  // 0..127
       const uint32_t conv0 = smem_u32(conv_smem);
+      // This thread's four chunks never change: chunk q of its four is row r = 16 q + ct / 8 (page q of the
+      // iteration, slot ct / 8), raw chunk c = ct % 8. Offsets inside a raw half-stage / an operand block:
+      const int rr = ct >> 3, c = ct & 7, sw = rr & 7;
+      const uint32_t src_off = static_cast<uint32_t>(rr * 128 + ((c ^ sw) << 4));          // + q * raw tile
+      const int line = c >> 2, c2 = (c & 3) * 2;
+      const uint32_t k_off = static_cast<uint32_t>(line * (64 * 128) + rr * 128);           // + q * 16 rows
+      const uint32_t v_off = static_cast<uint32_t>(kTcKBytes + line * (kPageSize * 128) + rr * 128);  // + q * V tile
+      const uint32_t ch0 = static_cast<uint32_t>((c2 ^ sw) << 4), ch1 = static_cast<uint32_t>(((c2 + 1) ^ sw) << 4);
       uint32_t slot = 0, slot_par = 0, stage_i = 0, stage_par = 0;
       bool ok = true;
       for (int it = 0; it < n_iters; ++it) {
         ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);                        // raw tiles have landed
-        if (ok && it >= C::kConvSlots) ok = mbar_wait_bounded(conv_free0 + 8 * slot, slot_par ^ 1);  // PV(it - 3) done
+        if (ok && it >= C::kConvSlots) ok = mbar_wait_bounded(conv_free0 + 8 * slot, slot_par ^ 1);  // PV(it - kConvSlots) done
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         const uint32_t raw = ring + stage_i * kTcStageBytes;
@@ -496,33 +508,24 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         const float* sc = scale_sh + stage_i * 8;
         const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
         const int valid_rows = min(L - (page0 + it * kTcPagesPerIter) * kPageSize, n_here * kPageSize);  // token rows of this block
-  #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const int idx = q4 * 128 + ct;            // chunk index: 64 rows x 8 chunks
-          const int r = idx >> 3, c = idx & 7;      // stacked token row (page r / 16, slot r % 16), raw chunk
-          const int pj = r >> 4, rr = r & 15;
-          if (pj < n_here) {
-            const uint32_t src_off = static_cast<uint32_t>(pj * C::kRawTileBytes + rr * 128 + ((c ^ (rr & 7)) << 4));
-            const int line = c >> 2, c2 = (c & 3) * 2;
-            // K: [line][64 rows][128 B], row r; V: page tile pj = [line][16 rows][128 B], row rr
-            const uint32_t k_dst = dst + line * (64 * 128) + r * 128;
-            const uint32_t v_dst = dst + kTcKBytes + pj * kTcTileBytes + line * (kPageSize * 128) + rr * 128;
-            const int sw = r & 7;  // (== rr & 7)
-            uint4 kin, vin, lo, hi;
-            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kin.x), "=r"(kin.y), "=r"(kin.z), "=r"(kin.w) : "r"(raw + src_off));
+#pragma unroll
+        for (int q = 0; q < kTcPagesPerIter; ++q) {
+          if (q < n_here) {  // (uniform)
+            uint4 kin, vin, klo, khi, vlo, vhi;
+            const uint32_t src = raw + q * C::kRawTileBytes + src_off;
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kin.x), "=r"(kin.y), "=r"(kin.z), "=r"(kin.w) : "r"(src));
             asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(vin.x), "=r"(vin.y), "=r"(vin.z), "=r"(vin.w)
-                         : "r"(raw + kTcPagesPerIter * C::kRawTileBytes + src_off));
-            const bool live = r < valid_rows;
-            const uint32_t ks2 = pack2<true>(sc[pj], sc[pj]);
-            const uint32_t vs2 = pack2<true>(sc[4 + pj], sc[4 + pj]);
-            e4m3x16_to_f16(kin, ks2, lo, hi);
-            if (!live) { lo = make_uint4(0u, 0u, 0u, 0u); hi = lo; }
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(k_dst + ((c2 ^ sw) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w));
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(k_dst + (((c2 + 1) ^ sw) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w));
-            e4m3x16_to_f16(vin, vs2, lo, hi);
-            if (!live) { lo = make_uint4(0u, 0u, 0u, 0u); hi = lo; }
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(v_dst + ((c2 ^ sw) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w));
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(v_dst + (((c2 + 1) ^ sw) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w));
+                         : "r"(src + kTcPagesPerIter * C::kRawTileBytes));
+            e4m3x16_to_f16(kin, pack2<true>(sc[q], sc[q]), klo, khi);
+            e4m3x16_to_f16(vin, pack2<true>(sc[4 + q], sc[4 + q]), vlo, vhi);
+            if (q * kPageSize + rr >= valid_rows) {  // a row past the end of the sequence (last block only)
+              klo = make_uint4(0u, 0u, 0u, 0u); khi = klo; vlo = klo; vhi = klo;
+            }
+            const uint32_t kd = dst + k_off + q * (kPageSize * 128), vd = dst + v_off + q * kTcTileBytes;
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(kd + ch0), "r"(klo.x), "r"(klo.y), "r"(klo.z), "r"(klo.w));
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(kd + ch1), "r"(khi.x), "r"(khi.y), "r"(khi.z), "r"(khi.w));
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(vd + ch0), "r"(vlo.x), "r"(vlo.y), "r"(vlo.z), "r"(vlo.w));
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(vd + ch1), "r"(vhi.x), "r"(vhi.y), "r"(vhi.z), "r"(vhi.w));
           }
         }
         fence_proxy_async();   // the tensor core reads the block through the async proxy
