@@ -158,6 +158,22 @@ def kv_append_e4m3(k_new, v_new, k_cache, v_cache, k_scale, v_scale, block_table
         C.c_int32(block_table.shape[1]), _p(seq_lens), C.c_int32(seq_lens.shape[0]))
 
 
+def kv_append_tokens_e4m3(k_new, v_new, k_cache, v_cache, k_scale, v_scale, block_table, seq_lens):
+    """In-place quantising append of ``k_new, v_new [B,T,Hkv,D]`` (bf16 bits): the one-token rule of
+    ``kv_append_e4m3`` applied to the block's tokens in order (``seq_lens`` = lengths after the append)."""
+    assert k_cache.dtype == np.uint8 and v_cache.dtype == np.uint8 and k_new.dtype == np.uint16
+    assert k_new.ndim == 4 and k_scale.dtype == np.float32 and k_scale.flags.c_contiguous and v_scale.flags.c_contiguous
+    k_new, v_new = np.ascontiguousarray(k_new), np.ascontiguousarray(v_new)
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    ps, hs, ss = _cache_strides(k_cache)
+    _, Hkv, P, D = k_cache.shape
+    _load().oracle_kv_append_tokens_e4m3(
+        _p(k_new), _p(v_new), _p(k_cache), _p(v_cache), _p(k_scale), _p(v_scale), C.c_int64(ps),
+        C.c_int64(hs), C.c_int64(ss), C.c_int32(P), C.c_int32(Hkv), C.c_int32(D), _p(block_table),
+        C.c_int32(block_table.shape[1]), _p(seq_lens), C.c_int32(seq_lens.shape[0]), C.c_int32(k_new.shape[1]))
+
+
 def paged_verify_attention(q, k_cache, v_cache, block_table, seq_lens, scale,
                            k_scale=None, v_scale=None, n_threads=0):
     """Causal attention of a block of query tokens: ``q [B,T,Hq,D]`` -> ``(out, lse)`` fp64;

@@ -262,6 +262,35 @@ void oracle_kv_append_tokens(const uint8_t* k_new, const uint8_t* v_new, uint8_t
 //   slot  > 0: scale[page,g] is the value stored when the page was opened;
 //   bytes = e4m3 nearest to x / scale (fp32 division, ties to the even code),
 //           saturating at +-448 (later rows may exceed the first row's range).
+// One row of the quantising append: the new bf16 row `src` becomes logical token `pos` of sequence b.
+static void append_row_e4m3(const uint16_t* src, uint8_t* cache, float* scales, int64_t page_stride,
+                            int64_t head_stride, int64_t slot_stride, int32_t page_size,
+                            int32_t num_kv_heads, int32_t head_dim, const int32_t* table_row,
+                            int64_t pos, int g, const double* pos_code) {
+  const int64_t page = table_row[pos / page_size];
+  const int64_t slot = pos % page_size;
+  float& sc = scales[page * num_kv_heads + g];
+  if (slot == 0) {
+    float amax = 0.0f;
+    for (int d = 0; d < head_dim; ++d) {
+      const float a = std::fabs(static_cast<float>(bf16_to_double(src[d])));
+      if (a > amax) amax = a;
+    }
+    sc = amax > 0.0f ? (amax * 2.0f) / 448.0f : 1.0f;
+  }
+  uint8_t* dst = cache + page * page_stride + g * head_stride + slot * slot_stride;
+  for (int d = 0; d < head_dim; ++d) {
+    const float y = static_cast<float>(bf16_to_double(src[d])) / sc;
+    const double a = std::fabs(static_cast<double>(y));
+    int best = 0;
+    for (int i = 1; i < 127; ++i) {
+      const double di = std::fabs(pos_code[i] - a), db = std::fabs(pos_code[best] - a);
+      if (di < db || (di == db && (i % 2 == 0))) best = i;
+    }
+    dst[d] = static_cast<uint8_t>(best | (std::signbit(y) ? 0x80 : 0));
+  }
+}
+
 void oracle_kv_append_e4m3(const uint16_t* k_new, const uint16_t* v_new, uint8_t* k_cache,
                            uint8_t* v_cache, float* k_scale, float* v_scale, int64_t page_stride,
                            int64_t head_stride, int64_t slot_stride, int32_t page_size,
@@ -272,34 +301,41 @@ void oracle_kv_append_e4m3(const uint16_t* k_new, const uint16_t* v_new, uint8_t
   for (int b = 0; b < batch; ++b) {
     const int64_t L = seq_lens[b];
     if (L <= 0) continue;
-    const int64_t page = block_table[static_cast<int64_t>(b) * block_table_stride + (L - 1) / page_size];
-    const int64_t slot = (L - 1) % page_size;
-    for (int which = 0; which < 2; ++which) {
-      const uint16_t* src_all = which ? v_new : k_new;
-      uint8_t* cache = which ? v_cache : k_cache;
-      float* scales = which ? v_scale : k_scale;
+    const int32_t* row = block_table + static_cast<int64_t>(b) * block_table_stride;
+    for (int g = 0; g < num_kv_heads; ++g) {
+      const int64_t src = (static_cast<int64_t>(b) * num_kv_heads + g) * head_dim;
+      append_row_e4m3(k_new + src, k_cache, k_scale, page_stride, head_stride, slot_stride, page_size,
+                      num_kv_heads, head_dim, row, L - 1, g, pos);
+      append_row_e4m3(v_new + src, v_cache, v_scale, page_stride, head_stride, slot_stride, page_size,
+                      num_kv_heads, head_dim, row, L - 1, g, pos);
+    }
+  }
+}
+
+// Quantising append of n_new tokens per sequence (rows [B, n_new, Hkv, D]): the one-token rule above
+// applied to token i = 0, 1, ... in this order, token i standing at position L_b - n_new + i -- so a
+// page opened inside the block takes its scale from the block's own row that lands in its slot 0.
+void oracle_kv_append_tokens_e4m3(const uint16_t* k_new, const uint16_t* v_new, uint8_t* k_cache,
+                                  uint8_t* v_cache, float* k_scale, float* v_scale,
+                                  int64_t page_stride, int64_t head_stride, int64_t slot_stride,
+                                  int32_t page_size, int32_t num_kv_heads, int32_t head_dim,
+                                  const int32_t* block_table, int32_t block_table_stride,
+                                  const int32_t* seq_lens, int32_t batch, int32_t n_new) {
+  double pos[127];
+  for (int i = 0; i < 127; ++i) pos[i] = e4m3_to_double(static_cast<uint8_t>(i));
+  for (int b = 0; b < batch; ++b) {
+    const int64_t L = seq_lens[b];
+    if (L <= 0) continue;
+    const int32_t* row = block_table + static_cast<int64_t>(b) * block_table_stride;
+    for (int i = 0; i < n_new; ++i) {
+      const int64_t at = L - n_new + i;
+      if (at < 0) continue;
       for (int g = 0; g < num_kv_heads; ++g) {
-        const uint16_t* src = src_all + (static_cast<int64_t>(b) * num_kv_heads + g) * head_dim;
-        float& sc = scales[page * num_kv_heads + g];
-        if (slot == 0) {
-          float amax = 0.0f;
-          for (int d = 0; d < head_dim; ++d) {
-            const float a = std::fabs(static_cast<float>(bf16_to_double(src[d])));
-            if (a > amax) amax = a;
-          }
-          sc = amax > 0.0f ? (amax * 2.0f) / 448.0f : 1.0f;
-        }
-        uint8_t* dst = cache + page * page_stride + g * head_stride + slot * slot_stride;
-        for (int d = 0; d < head_dim; ++d) {
-          const float y = static_cast<float>(bf16_to_double(src[d])) / sc;
-          const double a = std::fabs(static_cast<double>(y));
-          int best = 0;
-          for (int i = 1; i < 127; ++i) {
-            const double di = std::fabs(pos[i] - a), db = std::fabs(pos[best] - a);
-            if (di < db || (di == db && (i % 2 == 0))) best = i;
-          }
-          dst[d] = static_cast<uint8_t>(best | (std::signbit(y) ? 0x80 : 0));
-        }
+        const int64_t src = ((static_cast<int64_t>(b) * n_new + i) * num_kv_heads + g) * head_dim;
+        append_row_e4m3(k_new + src, k_cache, k_scale, page_stride, head_stride, slot_stride, page_size,
+                        num_kv_heads, head_dim, row, at, g, pos);
+        append_row_e4m3(v_new + src, v_cache, v_scale, page_stride, head_stride, slot_stride, page_size,
+                        num_kv_heads, head_dim, row, at, g, pos);
       }
     }
   }

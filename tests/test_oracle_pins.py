@@ -475,3 +475,51 @@ def test_e4m3_append_policy_against_library_cast(oracle):
     # a row 4x larger than the page's first row saturates at +-448 somewhere
     t = oracle.e4m3_decode_table()
     assert np.abs(t[kc[table[0, 0], :, 4]]).max() == 448.0
+
+
+def test_e4m3_block_append_is_the_one_token_rule_in_order(oracle):
+    """A block of T tokens appended at once must leave exactly what T one-token appends (pinned
+    above against the library cast) leave: same bytes, same scales, including pages opened inside
+    the block (their scale comes from the block's own row in slot 0) and sequences shorter than T."""
+    rng = np.random.default_rng(11)
+    Hkv, D, P, T = 2, 64, 16, 7
+    n_pages = 8
+    table = np.array([[2, 0, 5], [3, 1, 6], [4, 7, 0]], np.int32)
+    final = np.array([21, 16, 3], np.int32)       # crosses a page boundary / ends on one / shorter than the block
+    kn = W.f32_to_bf16_bits((rng.standard_normal((3, T, Hkv, D)) * 2).astype(np.float32))
+    vn = W.f32_to_bf16_bits(rng.standard_normal((3, T, Hkv, D)).astype(np.float32))
+
+    def fresh():
+        kc = np.full((n_pages, Hkv, P, D), 0xFF, np.uint8)
+        ks = np.full((n_pages, Hkv), np.nan, np.float32)
+        return kc, kc.copy(), ks, ks.copy()
+
+    # history before the block: one-token appends up to final - T
+    kc, vc, ks, vs = fresh()
+    kc2, vc2, ks2, vs2 = fresh()
+    for step in range(int((final - T).max())):
+        lens = np.minimum(step + 1, np.maximum(final - T, 0)).astype(np.int32)
+        if step >= lens.max():
+            break
+        hk = W.f32_to_bf16_bits(np.random.default_rng(100 + step).standard_normal((3, Hkv, D)).astype(np.float32))
+        hv = W.f32_to_bf16_bits(np.random.default_rng(200 + step).standard_normal((3, Hkv, D)).astype(np.float32))
+        active = (step + 1) <= np.maximum(final - T, 0)
+        lens = np.where(active, step + 1, 0).astype(np.int32)      # length 0: no append for that sequence
+        for args in ((kc, vc, ks, vs), (kc2, vc2, ks2, vs2)):
+            oracle.kv_append_e4m3(hk, hv, args[0], args[1], args[2], args[3], table, lens)
+    # the block at once ...
+    oracle.kv_append_tokens_e4m3(kn, vn, kc, vc, ks, vs, table, final)
+    # ... against token by token
+    for i in range(T):
+        at = final - T + i                          # position of token i
+        lens = np.where(at >= 0, at + 1, 0).astype(np.int32)
+        oracle.kv_append_e4m3(np.ascontiguousarray(kn[:, i]), np.ascontiguousarray(vn[:, i]),
+                              kc2, vc2, ks2, vs2, table, lens)
+    assert (kc == kc2).all() and (vc == vc2).all()
+    assert np.array_equal(ks, ks2, equal_nan=True) and np.array_equal(vs, vs2, equal_nan=True)
+    # a block of one token is the one-token append
+    a, b = fresh(), fresh()
+    lens1 = np.array([1, 17, 5], np.int32)
+    oracle.kv_append_tokens_e4m3(kn[:, :1], vn[:, :1], a[0], a[1], a[2], a[3], table, lens1)
+    oracle.kv_append_e4m3(np.ascontiguousarray(kn[:, 0]), np.ascontiguousarray(vn[:, 0]), b[0], b[1], b[2], b[3], table, lens1)
+    assert (a[0] == b[0]).all() and (a[1] == b[1]).all()
