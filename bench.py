@@ -233,7 +233,7 @@ def run_gpu(args):
             mc = pda.max_chunks(int(w.seq_lens.max()), chunk)
             vpo = torch.empty((w.batch, T, w.num_q_heads, mc, w.head_dim), dtype=torch.float32, device=dev)
             vpl = torch.empty((w.batch, T, w.num_q_heads, mc), dtype=torch.float32, device=dev)
-        launches_per_step = (2 if w.kv_dtype == "bf16" else 1) + (1 if chunk else 0)
+        launches_per_step = 2 + (1 if chunk else 0)
 
     def step(ev=None):
         if mode == "cascade":
@@ -248,8 +248,10 @@ def run_gpu(args):
                 ev[1].record(stream)
             return
         if mode == "verify":
-            if w.kv_dtype == "bf16":   # (there is no multi-token quantising append: e4m3 caches are attended as they are)
+            if w.kv_dtype == "bf16":
                 pda.kv_append_tokens(vk, vv, k_cache, v_cache, bt, sl, status=status)
+            else:
+                pda.kv_append_tokens_fp8(vk, vv, k_cache, v_cache, k_scale, v_scale, bt, sl, status=status)
             if ev:
                 ev[0].record(stream)
             pda.paged_verify_attention(vq, k_cache, v_cache, bt, sl, float(w.scale), chunk_tokens=chunk,

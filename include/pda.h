@@ -189,6 +189,18 @@ int kv_append_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_c
                   const int32_t* block_table, int32_t block_table_stride,
                   const int32_t* seq_lens, int32_t batch, int32_t* status, pda_stream_t stream);
 
+/* The same for a block of n_new tokens per sequence (the draft block of a
+ * verification step on an e4m3 cache): k_new, v_new are
+ * [batch, n_new, num_kv_heads, head_dim] bf16, token i becomes logical token
+ * seq_lens[b] - n_new + i, and the one-token rule above is applied to the tokens
+ * in this order -- a page opened inside the block takes its scale from the
+ * block's own row that lands in its slot 0. n_new == 1 is kv_append_fp8. */
+int kv_append_tokens_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                         const pda_cache_desc* desc, float* k_scale, float* v_scale,
+                         const int32_t* block_table, int32_t block_table_stride,
+                         const int32_t* seq_lens, int32_t batch, int32_t n_new, int32_t* status,
+                         pda_stream_t stream);
+
 /* Verification attention over a block of n_query_tokens draft tokens per sequence
  * (the predicted-output verifier of the paper scores 16-token blocks in one pass:
  * Section 4.2 and Appendix A, Scenario B; the paper prints no formula -- this is

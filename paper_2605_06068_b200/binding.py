@@ -24,7 +24,7 @@ EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "paged_decode_attention", "paged_decode_reduce", "paged_decode_step_host",
            "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
            "paged_decode_step", "pda_advance_seq_lens", "paged_window_decode_attention", "kv_append_tokens",
-           "paged_verify_attention", "paged_prefix_decode_attention", "kv_append_fp8",
+           "paged_verify_attention", "paged_prefix_decode_attention", "kv_append_fp8", "kv_append_tokens_fp8",
            "pda_set_persistent_threshold"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
@@ -61,6 +61,7 @@ def lib():
         L.pda_workspace_ints.argtypes = [i32, i32]
         L.pda_set_persistent_threshold.argtypes = [i32]
         L.kv_append_fp8.argtypes = [vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, vp, vp]
+        L.kv_append_tokens_fp8.argtypes = [vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, vp, vp]
         L.kv_append_tokens.argtypes = [vp, vp, vp, vp, dp, vp, i32, vp, i32, i32, vp, vp]
         L.paged_verify_attention.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, i32, f32,
                                              i32, vp, vp, vp, i32, u32, vp, vp]
@@ -332,6 +333,18 @@ def kv_append_fp8(k_new, v_new, k_cache, v_cache, k_scale, v_scale, block_table,
                              _ptr(k_scale), _ptr(v_scale), _ptr(block_table), block_table.stride(0),
                              _ptr(seq_lens), seq_lens.shape[0], _ptr(status), _stream(stream))
     _check(rc, "kv_append_fp8")
+
+
+def kv_append_tokens_fp8(k_new, v_new, k_cache, v_cache, k_scale, v_scale, block_table, seq_lens,
+                         status=None, stream=None):
+    """Quantising append of a block ``k_new, v_new [B,T,Hkv,D]`` bf16 into e4m3 caches."""
+    desc = cache_desc(k_cache)
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_scale.is_contiguous() and k_new.dim() == 4
+    rc = lib().kv_append_tokens_fp8(_ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), C.byref(desc),
+                                    _ptr(k_scale), _ptr(v_scale), _ptr(block_table), block_table.stride(0),
+                                    _ptr(seq_lens), seq_lens.shape[0], k_new.shape[1], _ptr(status),
+                                    _stream(stream))
+    _check(rc, "kv_append_tokens_fp8")
 
 
 def set_persistent_threshold(min_units_per_cta: int):

@@ -251,15 +251,16 @@ int kv_append_tokens(const void* k_new, const void* v_new, void* k_cache, void* 
                                                        static_cast<cudaStream_t>(stream)));
 }
 
-int kv_append_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
-                  const pda_cache_desc* desc, float* k_scale, float* v_scale,
-                  const int32_t* block_table, int32_t block_table_stride,
-                  const int32_t* seq_lens, int32_t batch, int32_t* status, pda_stream_t stream) {
+namespace {
+int append_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+               const pda_cache_desc* desc, float* k_scale, float* v_scale, const int32_t* block_table,
+               int32_t block_table_stride, const int32_t* seq_lens, int32_t batch, int32_t n_new,
+               int32_t* status, pda_stream_t stream) {
   CacheGeom g;
   if (int rc = check_desc(desc, &g)) return rc;
   if (g.dtype != PDA_FP8_E4M3 || g.head_dim % 64 != 0) return PDA_ERR_UNSUPPORTED;
-  if (batch < 0 || block_table_stride < 0) return PDA_ERR_INVALID_ARG;
-  if (batch == 0) return PDA_OK;
+  if (batch < 0 || block_table_stride < 0 || n_new < 0) return PDA_ERR_INVALID_ARG;
+  if (batch == 0 || n_new == 0) return PDA_OK;
   if (!k_new || !v_new || !k_cache || !v_cache || !k_scale || !v_scale || !block_table ||
       !seq_lens || block_table_stride == 0)
     return PDA_ERR_INVALID_ARG;
@@ -267,8 +268,26 @@ int kv_append_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_c
     return PDA_ERR_MISALIGNED;
   return static_cast<int>(pda::launch_kv_append_e4m3(k_new, v_new, k_cache, v_cache, k_scale,
                                                      v_scale, g, block_table, block_table_stride,
-                                                     seq_lens, batch, status,
+                                                     seq_lens, batch, n_new, status,
                                                      static_cast<cudaStream_t>(stream)));
+}
+}  // namespace
+
+int kv_append_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                  const pda_cache_desc* desc, float* k_scale, float* v_scale,
+                  const int32_t* block_table, int32_t block_table_stride,
+                  const int32_t* seq_lens, int32_t batch, int32_t* status, pda_stream_t stream) {
+  return append_fp8(k_new, v_new, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                    block_table_stride, seq_lens, batch, 1, status, stream);
+}
+
+int kv_append_tokens_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                         const pda_cache_desc* desc, float* k_scale, float* v_scale,
+                         const int32_t* block_table, int32_t block_table_stride,
+                         const int32_t* seq_lens, int32_t batch, int32_t n_new, int32_t* status,
+                         pda_stream_t stream) {
+  return append_fp8(k_new, v_new, k_cache, v_cache, desc, k_scale, v_scale, block_table,
+                    block_table_stride, seq_lens, batch, n_new, status, stream);
 }
 
 int paged_verify_attention(const void* q, const void* k_cache, const void* v_cache,

@@ -93,7 +93,7 @@ cudaError_t launch_kv_append(const void* k_new, const void* v_new, void* k_cache
 cudaError_t launch_kv_append_e4m3(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                   float* k_scale, float* v_scale, const CacheGeom& g,
                                   const int32_t* block_table, int32_t bt_stride,
-                                  const int32_t* seq_lens, int32_t batch, int32_t* status,
+                                  const int32_t* seq_lens, int32_t batch, int32_t n_new, int32_t* status,
                                   cudaStream_t stream);
 cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t delta, cudaStream_t stream);
 cudaError_t launch_attention_generic(const AttnParams& p, cudaStream_t stream);

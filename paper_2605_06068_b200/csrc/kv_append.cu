@@ -99,13 +99,16 @@ cudaError_t launch_kv_append_tokens(const void* k_new, const void* v_new, void* 
 // Quantising append into an e4m3 cache: one warp per (sequence, kv head, K|V). The page's
 // scale is fixed by its first row (amax * 2 / 448, or 1 for an all-zero row); later rows reuse
 // it and saturate at +-448. x / scale is an IEEE fp32 division, the cast rounds to nearest even.
+// One warp per (sequence, kv head, K | V) walks the block's n_new tokens in order, so that a page opened
+// inside the block gets its scale from the block's own row in slot 0 before the later rows use it (the
+// scale of the page being filled stays in a register; a page opened by an earlier call is read once).
 __global__ void kv_append_e4m3_kernel(const __nv_bfloat16* __restrict__ k_new,
                                       const __nv_bfloat16* __restrict__ v_new,
                                       uint8_t* __restrict__ k_cache, uint8_t* __restrict__ v_cache,
                                       float* __restrict__ k_scale, float* __restrict__ v_scale,
                                       CacheGeom g, const int32_t* __restrict__ block_table,
                                       int32_t bt_stride, const int32_t* __restrict__ seq_lens,
-                                      int32_t batch, int32_t* status) {
+                                      int32_t batch, int32_t n_new, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int64_t unit = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
   if (unit >= 2ll * batch * g.num_kv_heads) return;
@@ -118,40 +121,48 @@ __global__ void kv_append_e4m3_kernel(const __nv_bfloat16* __restrict__ k_new,
     if (lane == 0) report(status, PDA_DEV_BAD_SEQ_LEN);
     return;
   }
-  const int page = block_table[static_cast<int64_t>(b) * bt_stride + (L - 1) / kPageSize];
-  if (page < 0 || page >= g.num_pages) {
-    if (lane == 0) report(status, PDA_DEV_BAD_PAGE);
-    return;
-  }
-  const int slot = (L - 1) % kPageSize;
   const int per_lane = g.head_dim / 32;  // 2, 4, 6 or 8 consecutive elements
-  const __nv_bfloat16* src = (is_v ? v_new : k_new) + r * g.head_dim + lane * per_lane;
-  float x[8];
-  float amax = 0.f;
+  int cur_page = -1;   // the page whose scale `sc` is
+  float sc = 1.f;
+  for (int i = 0; i < n_new; ++i) {
+    const int pos = L - n_new + i;
+    if (pos < 0) continue;
+    const int page = block_table[static_cast<int64_t>(b) * bt_stride + pos / kPageSize];
+    if (page < 0 || page >= g.num_pages) {
+      if (lane == 0) report(status, PDA_DEV_BAD_PAGE);
+      cur_page = -1;
+      continue;
+    }
+    const int slot = pos % kPageSize;
+    const __nv_bfloat16* src = (is_v ? v_new : k_new) +
+                               ((static_cast<int64_t>(b) * n_new + i) * g.num_kv_heads + head) * g.head_dim + lane * per_lane;
+    float x[8];
+    float amax = 0.f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    x[i] = i < per_lane ? __bfloat162float(src[i]) : 0.f;
-    amax = fmaxf(amax, fabsf(x[i]));
-  }
-  float* scale_ptr = (is_v ? v_scale : k_scale) + static_cast<int64_t>(page) * g.num_kv_heads + head;
-  float sc;
-  if (slot == 0) {
+    for (int e = 0; e < 8; ++e) {
+      x[e] = e < per_lane ? __bfloat162float(src[e]) : 0.f;
+      amax = fmaxf(amax, fabsf(x[e]));
+    }
+    float* scale_ptr = (is_v ? v_scale : k_scale) + static_cast<int64_t>(page) * g.num_kv_heads + head;
+    if (slot == 0) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    sc = amax > 0.f ? __fdiv_rn(amax * 2.0f, 448.0f) : 1.0f;
-    if (lane == 0) *scale_ptr = sc;
-  } else {
-    sc = *scale_ptr;
-  }
-  uint8_t* dst = (is_v ? v_cache : k_cache) + page * g.page_stride + head * g.head_stride +
-                 slot * g.slot_stride + lane * per_lane;
+      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      sc = amax > 0.f ? __fdiv_rn(amax * 2.0f, 448.0f) : 1.0f;
+      if (lane == 0) *scale_ptr = sc;
+    } else if (page != cur_page) {
+      sc = *scale_ptr;   // opened by an earlier call
+    }
+    cur_page = page;
+    uint8_t* dst = (is_v ? v_cache : k_cache) + page * g.page_stride + head * g.head_stride +
+                   slot * g.slot_stride + lane * per_lane;
 #pragma unroll
-  for (int i = 0; i < 8; i += 2) {
-    if (i < per_lane) {
-      uint16_t packed;
-      const float lo = __fdiv_rn(x[i], sc), hi = __fdiv_rn(x[i + 1], sc);
-      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(packed) : "f"(hi), "f"(lo));
-      *reinterpret_cast<uint16_t*>(dst + i) = packed;
+    for (int e = 0; e < 8; e += 2) {
+      if (e < per_lane) {
+        uint16_t packed;
+        const float lo = __fdiv_rn(x[e], sc), hi = __fdiv_rn(x[e + 1], sc);
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(packed) : "f"(hi), "f"(lo));
+        *reinterpret_cast<uint16_t*>(dst + e) = packed;
+      }
     }
   }
 }
@@ -159,16 +170,16 @@ __global__ void kv_append_e4m3_kernel(const __nv_bfloat16* __restrict__ k_new,
 cudaError_t launch_kv_append_e4m3(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                   float* k_scale, float* v_scale, const CacheGeom& g,
                                   const int32_t* block_table, int32_t bt_stride,
-                                  const int32_t* seq_lens, int32_t batch, int32_t* status,
+                                  const int32_t* seq_lens, int32_t batch, int32_t n_new, int32_t* status,
                                   cudaStream_t stream) {
   const int64_t warps = 2ll * batch * g.num_kv_heads;
-  if (warps == 0) return cudaSuccess;
+  if (warps == 0 || n_new == 0) return cudaSuccess;
   const int threads = 128;
   const unsigned blocks = static_cast<unsigned>((warps * 32 + threads - 1) / threads);
   kv_append_e4m3_kernel<<<blocks, threads, 0, stream>>>(
       static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
       static_cast<uint8_t*>(k_cache), static_cast<uint8_t*>(v_cache), k_scale, v_scale, g,
-      block_table, bt_stride, seq_lens, batch, status);
+      block_table, bt_stride, seq_lens, batch, n_new, status);
   return cudaGetLastError();
 }
 

@@ -592,3 +592,56 @@ def test_fp8_append_bit_exact_and_attention_on_the_grown_cache(oracle, shape):
     out = pda.paged_decode_attention(bf16_tensor(q), dk, dv, bt, torch.from_numpy(lens).cuda(),
                                      float(np.float32(1 / np.sqrt(D))), k_scale=dks, v_scale=dvs, status=status)
     assert_close(bf16_to_f64(out), ref, "e4m3", what="attention after fp8 appends")
+
+
+@pytest.mark.parametrize("shape", [(8, 2, 64), (32, 8, 128)])
+def test_fp8_block_append_bit_exact_and_verified(oracle, shape):
+    """Blocks of T tokens quantised into e4m3 caches: bytes and scales equal the oracle's (which is the
+    one-token rule in order), over several blocks that open pages in their middle, start from empty
+    sequences and include a sequence shorter than a block; then the block is verified over that cache."""
+    Hq, Hkv, D = shape
+    B, T, n_blocks = 4, 7, 5
+    rng = np.random.default_rng(21)
+    first = np.array([7, 20, 3, 16], np.int32)      # lengths after the first block (3 < T: partial block)
+    max_len = int(first.max()) + T * (n_blocks - 1)
+    pages_per_seq = (max_len + 15) // 16
+    n_pages = B * pages_per_seq + 2
+    table = rng.permutation(n_pages)[:B * pages_per_seq].reshape(B, pages_per_seq).astype(np.int32)
+    hk = np.full((n_pages, Hkv, 16, D), 0xFF, np.uint8); hv = hk.copy()
+    hks = np.full((n_pages, Hkv), np.nan, np.float32); hvs = hks.copy()
+    # sequence 1 has 13 earlier tokens (so that its first block lands in the middle of a page it did not open)
+    pre = np.array([0, 13, 0, 9], np.int32)
+    for t in range(int(pre.max())):
+        cur = np.where(t < pre, t + 1, 0).astype(np.int32)
+        kn1 = W.f32_to_bf16_bits(rng.standard_normal((B, Hkv, D)).astype(np.float32))
+        vn1 = W.f32_to_bf16_bits(rng.standard_normal((B, Hkv, D)).astype(np.float32))
+        oracle.kv_append_e4m3(kn1, vn1, hk, hv, hks, hvs, table, cur)
+    dk, dv = torch.from_numpy(hk.copy()).cuda(), torch.from_numpy(hv.copy()).cuda()
+    dks, dvs = torch.from_numpy(hks.copy()).cuda(), torch.from_numpy(hvs.copy()).cuda()
+    bt = torch.from_numpy(table).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lens = first.copy()
+    for blk in range(n_blocks):
+        amp = 1.0 + 4.0 * (blk == 2)
+        kn = W.f32_to_bf16_bits((rng.standard_normal((B, T, Hkv, D)) * amp).astype(np.float32))
+        vn = W.f32_to_bf16_bits(rng.standard_normal((B, T, Hkv, D)).astype(np.float32))
+        oracle.kv_append_tokens_e4m3(kn, vn, hk, hv, hks, hvs, table, lens)
+        pda.kv_append_tokens_fp8(bf16_tensor(kn), bf16_tensor(vn), dk, dv, dks, dvs, bt,
+                                 torch.from_numpy(lens).cuda(), status=status)
+        assert (dk.cpu().numpy() == hk).all() and (dv.cpu().numpy() == hv).all(), f"block {blk}"
+        gks, gvs = dks.cpu().numpy(), dvs.cpu().numpy()
+        live = ~np.isnan(hks)
+        assert (np.isnan(gks) == np.isnan(hks)).all() and (gks[live] == hks[live]).all() and (gvs[live] == hvs[live]).all()
+        if blk < n_blocks - 1:
+            lens = lens + T
+    assert int(status.item()) == 0
+    if D != 128:
+        return      # multi-query attention over e4m3 caches is built for head_dim 128
+    # the last block's queries over the cache that now holds it
+    scale = np.float32(1 / np.sqrt(D))
+    q = W.f32_to_bf16_bits(rng.standard_normal((B, T, Hq, D), dtype=np.float32))
+    ref, _ = oracle.paged_verify_attention(q, hk, hv, table, lens, scale, hks, hvs)
+    out = pda.paged_verify_attention(bf16_tensor(q), dk, dv, bt, torch.from_numpy(lens).cuda(), float(scale),
+                                     k_scale=dks, v_scale=dvs, status=status)
+    assert_close(bf16_to_f64(out), ref, "e4m3", what="verify after fp8 block appends")
+    assert int(status.item()) == 0
