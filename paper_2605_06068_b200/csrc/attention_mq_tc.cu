@@ -1,12 +1,7 @@
-// Multi-query paged attention on the 5th-generation tensor cores (tcgen05 + TMEM),
-// bf16 KV with head_dim 128 or 64 (the figures in this comment are for 128), or e4m3 KV with head_dim
-// 128. The tensor core has no bf16 x e4m3 mode and e4m3 x e4m3 would quantise Q and P, so e4m3 tiles are
-// converted: the TMA ring holds the raw tiles, four converter warps write them as f16 operand blocks
-// (exact conversion, the page's scale folded in, rows past the sequence end zeroed) into three
-// conversion slots, and Q, P and the tile of ones are f16 as well. That variant runs 16 warps as four
-// warpgroups and redistributes registers between them (setmaxnreg). Same contract as attention_mq.cu (verification of a
-// block of draft tokens; the shared-prefix part of a decode batch): up to 128
-// query rows (query tokens x group size) per CTA against one sequence's pages.
+// Multi-query paged attention on the 5th-generation tensor cores (tcgen05 + TMEM): verification of a
+// block of draft tokens, and the shared-prefix part of a decode batch; same contract as attention_mq.cu.
+// Up to 128 query rows (query tokens x group size) per CTA against one sequence's pages. bf16 KV with
+// head_dim 128 or 64 (the figures in this comment are for 128), or e4m3 KV with head_dim 128.
 //
 // This is the part of the path that is a real dense contraction, so it runs as
 // UMMA tiles with operands and accumulators in tensor memory (TMEM, 128 lanes = query rows):
@@ -40,6 +35,12 @@
 //               TMEM when the max grew by more than 2^8 -> wait PV(i-2) (P buffer free) -> P =
 //               exp2(S * scale - ref) as bf16 pairs (packed f32x2 FMA, one exp2 per element) ->
 //               tcgen05.st P -> arrive(bar_p[i&1])
+// e4m3 KV: the tensor core has no bf16 x e4m3 mode and e4m3 x e4m3 would quantise Q and P, so the tiles
+// are converted. The TMA ring holds the raw tiles (128-byte rows), four converter warps (8-11) write
+// each iteration's K and V as an f16 operand block (exact conversion, the page's scale folded in, rows
+// past the sequence end zeroed) into one of three conversion slots, and Q, P and the tile of ones are
+// f16 as well. That variant runs 16 warps (producer 12, S issue 13, PV issue 14) as four warpgroups and
+// moves registers from the converter and control groups to the softmax groups (setmaxnreg).
 // All mbarrier waits are bounded; TMEM is always released before the CTA exits.
 #include "common.cuh"
 #include "tma_ptx.cuh"
