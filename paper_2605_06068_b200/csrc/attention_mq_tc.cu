@@ -53,41 +53,43 @@ constexpr int kTcRows = 128;            // query rows per CTA (UMMA M)
 constexpr int kTcPagesPerIter = 4;      // 64 tokens per iteration
 constexpr int kTcOnesBytes = 2048;                         // bf16 ones: B operand [16 tokens][16 columns] of the row-sum MMA
 constexpr int kTcMBytes = 2 * kTcRows * 4;                 // running row maxima handed between the two softmax sets
-// Sizes that depend on head_dim D (128 or 64) and on the cache's element type. A 16-bit row is D / 64
-// lines of 128 bytes. An operand block = what the tensor core reads for one iteration: K of 4 pages as
-// [lines][64 tokens][128 B], then 4 V page tiles. bf16 caches: the TMA ring holds operand blocks. e4m3
-// caches (D = 128): the ring holds the raw tiles (128-byte rows) and four converter warps turn them into
-// f16 operand blocks, exactly and with the page's scales folded in, in kConvSlots conversion slots.
+constexpr int kTcRowBytes = 3 * kTcRows * 4;               // e4m3: per-row score constant, the two sets' row sums
+// Sizes that depend on head_dim D (128 or 64) and on the cache's element size (e4m3: D = 128). A row of
+// the cache is D * element size / 128 lines of 128 bytes. An operand block = what the tensor core reads
+// for one iteration and what one ring stage holds: K of 4 pages as [lines][64 tokens][128 B], then 4 V
+// page tiles.
 template <int D, bool kFp8>
 struct TcCfg {
   static_assert(!kFp8 || D == 128, "e4m3 is built for head_dim 128");
-  static constexpr int kLines = D / 64;
-  static constexpr int kTileBytes = kPageSize * D * 2;          // one 16-bit K or V page tile: 4096 / 2048
-  static constexpr int kKBytes = kTcPagesPerIter * kTileBytes;  // K of 4 pages as [lines][64 tokens][128 B]
-  static constexpr int kOperandBytes = 2 * kKBytes;             // K block, then 4 V page tiles: 32 / 16 KB
-  static constexpr int kRawTileBytes = kPageSize * D;           // one e4m3 page tile: 2048
-  static constexpr int kStageBytes = kFp8 ? 2 * kTcPagesPerIter * kRawTileBytes : kOperandBytes;
-  static constexpr int kStages = kFp8 ? 6 : 6 * 128 / D;        // 192 KB of ring for 16-bit caches, 96 KB for e4m3
-  // (a slot is free again after the PV that read it; four slots with four raw stages, and separate pools
-  // for K and V, were measured no faster: the converters' instructions share the schedulers with the
-  // softmax warps, which is what stretches an iteration from 0.72 to 1.0 us)
-  static constexpr int kConvSlots = kFp8 ? 3 : 0;
-  static constexpr int kScaleBytes = kFp8 ? kStages * 2 * kTcPagesPerIter * 4 : 0;  // per stage: 4 K and 4 V scales
-  static constexpr int kSmemBytes = kStages * kStageBytes + kConvSlots * kOperandBytes + kTcOnesBytes + kTcMBytes +
-                                    kScaleBytes + 512 + 1024;
-  // warps: softmax 0-7; then (e4m3: converters 8-11) producer, S issue (+ TMEM allocation), PV issue
-  static constexpr int kProducerWarp = kFp8 ? 12 : 8, kMmaWarp = kProducerWarp + 1, kPvWarp = kProducerWarp + 2;
-  static constexpr int kThreads = kFp8 ? 512 : 352;
+  static constexpr int kElemBytes = kFp8 ? 1 : 2;
+  static constexpr int kLines = D * kElemBytes / 128;
+  static constexpr int kTileBytes = kPageSize * D * kElemBytes;  // one K or V page tile: 4096 / 2048 (bf16), 2048 (e4m3)
+  static constexpr int kKBytes = kTcPagesPerIter * kTileBytes;   // K of 4 pages as [lines][64 tokens][128 B]
+  static constexpr int kOperandBytes = 2 * kKBytes;              // K block, then 4 V page tiles: 32 / 16 KB
+  static constexpr int kStageBytes = kOperandBytes;
+  static constexpr int kStages = 192 * 1024 / kStageBytes;       // 192 KB in flight per SM
+  static constexpr int kScaleBytes = kFp8 ? kStages * 16 * 4 : 0;  // per stage and page: score factor, log2 and 1 / V scale
+  static constexpr int kSmemBytes = kStages * kStageBytes + kTcOnesBytes + kTcMBytes + kTcRowBytes + kScaleBytes +
+                                    512 + 1024;
+  // warps: softmax 0-7, producer, S issue (+ TMEM allocation), PV issue
+  static constexpr int kProducerWarp = 8, kMmaWarp = 9, kPvWarp = 10;
+  // e4m3: a twelfth, idle warp completes the third warpgroup, whose registers go to the softmax warps
+  static constexpr int kThreads = kFp8 ? 384 : 352;
 };
 constexpr int kTcSoftmaxWarps = 8;      // two sets of 4: set x takes the iterations it with it % 2 == x
-// e4m3 variant: four warpgroups whose registers are redistributed at the start (setmaxnreg):
-// 2 x 128 x 176 (softmax) + 128 x 80 (converters) + 128 x 64 (producer, issuers, one spare warp) <= 65536
-constexpr uint32_t kTcRegsSoftmax = 176, kTcRegsConvert = 80, kTcRegsControl = 64;
+// e4m3: three warpgroups start with 168 registers a thread; the control group keeps 72 and each softmax
+// group takes 208 (setmaxnreg): 2 x 128 x 208 + 128 x 72 <= 65536. With 168 the softmax loop spilled.
+constexpr uint32_t kTcRegsSoftmax = 208, kTcRegsControl = 72;
 // Tensor memory columns (32-bit each, 128 lanes = query rows): S buffers 0..63 and 64..127 (f32),
-// O 128..255 (f32), Q 256..319 (bf16 pairs along d), P buffers 320..351 and 352..383 (bf16 pairs
-// along tokens). Allocations are powers of two.
+// O 128..255 (f32), Q 256..319 (bf16 pairs along d; e4m3: the high parts in 256..287, four to a column,
+// the low parts in 288..319), P buffers 320..351 and 352..383 (bf16 pairs along tokens; e4m3: 16 columns
+// of high parts, then 16 of low parts). Allocations are powers of two.
+// e4m3: each softmax set accumulates into an O of its own (128..255 and 256..383; the two are merged at
+// the end like split-KV partials), Q 384..447, P buffers 448..479 and 480..511.
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kTmemO = 128, kTmemQ = 256, kTmemP = 320, kTmemL = 384;  // l: row sums of P, 16 columns (all equal)
+constexpr uint32_t kTmemO = 128, kTmemL = 384;  // l (bf16): row sums of P, 16 columns (all equal)
+template <bool kFp8> constexpr uint32_t kTmemQ = kFp8 ? 384 : 256;
+template <bool kFp8> constexpr uint32_t kTmemP = kFp8 ? 448 : 320;
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the max grows this much
 
 // Spinning bounded wait (no suspension): the waits on the MMA/softmax hand-off are short and on the
@@ -103,13 +105,22 @@ __device__ __forceinline__ void mbar_arrive_tc(uint32_t bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // D[tmem] (+)= A[tmem] . B[smem descriptor]; accumulate == 0 overwrites D. A is read from tensor memory
-// (lane = row, 32-bit column = two consecutive k elements).
+// (lane = row, 32-bit column = two consecutive 16-bit k elements, or four 8-bit ones). k8: both operands
+// e4m3, K = 32 per instruction; else bf16, K = 16.
+template <bool k8>
 __device__ __forceinline__ void tc_mma_ts_if(uint32_t leader, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
                                              uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred pe, pa;\n\tsetp.ne.b32 pe, %5, 0;\n\tsetp.ne.b32 pa, %4, 0;\n\t"
-      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pa;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
+  if constexpr (k8) {
+    asm volatile(
+        "{\n\t.reg .pred pe, pa;\n\tsetp.ne.b32 pe, %5, 0;\n\tsetp.ne.b32 pa, %4, 0;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, pa;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred pe, pa;\n\tsetp.ne.b32 pe, %5, 0;\n\tsetp.ne.b32 pa, %4, 0;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pa;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
+  }
 }
 __device__ __forceinline__ void tc_commit_if(uint32_t leader, uint32_t bar) {
   asm volatile(
@@ -124,24 +135,34 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lbo_byt
          (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) |
          (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: f32 accumulate, A and B both bf16 or both f16, A K-major, M = 128.
-__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major, bool f16) {
-  return (1u << 4) | ((f16 ? 0u : 1u) << 7) | ((f16 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+// Instruction descriptor: f32 accumulate, A K-major, M = 128; A and B both bf16 (kind::f16, format 1) or
+// both e4m3 (kind::f8f6f4, format 0).
+__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major, bool e4m3) {
+  return (1u << 4) | ((e4m3 ? 0u : 1u) << 7) | ((e4m3 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) |
          (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTcRows >> 4) << 24);
 }
 template <uint32_t kRegs>
 __device__ __forceinline__ void reg_alloc_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs)); }
 template <uint32_t kRegs>
 __device__ __forceinline__ void reg_alloc_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs)); }
-// 16 e4m3 values (one 16-byte chunk) -> 16 f16 values times a scale, as two 16-byte chunks
-__device__ __forceinline__ void e4m3x16_to_f16(const uint4& in, uint32_t scale2, uint4& lo, uint4& hi) {
-  auto cv = [&](uint32_t w, uint32_t& a, uint32_t& b) {
-    a = e4m3x2_to_f16x2(w & 0xffffu);
-    b = e4m3x2_to_f16x2(w >> 16);
-    asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(a) : "r"(scale2));
-    asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b) : "r"(scale2));
-  };
-  cv(in.x, lo.x, lo.y); cv(in.y, lo.z, lo.w); cv(in.z, hi.x, hi.y); cv(in.w, hi.z, hi.w);
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// Two f32 -> two e4m3 bytes (lo in bits 0..7), round to nearest, saturating.
+__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// x = hi + lo with both parts e4m3: hi keeps the top three mantissa bits of x (exact in e4m3 from 2^-6
+// up), lo is the remainder rounded. |x - hi - lo| <= max(2^-7 |x|, 2^-10); 0 <= x <= 448 or so.
+__device__ __forceinline__ void split_e4m3x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const float t0 = __uint_as_float(__float_as_uint(x0) & 0xfff00000u);
+  const float t1 = __uint_as_float(__float_as_uint(x1) & 0xfff00000u);
+  hi = f32x2_to_e4m3x2(t0, t1);
+  lo = f32x2_to_e4m3x2(x0 - t0, x1 - t1);
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -180,6 +201,11 @@ __device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   return d;
 }
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -194,13 +220,14 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   constexpr int kTcProducerWarp = C::kProducerWarp, kTcMmaWarp = C::kMmaWarp, kTcPvWarp = C::kPvWarp;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* conv_smem = smem + kTcStages * kTcStageBytes;             // e4m3: kConvSlots operand blocks
-  uint8_t* ones_smem = conv_smem + C::kConvSlots * C::kOperandBytes;
+  uint8_t* ones_smem = smem + kTcStages * kTcStageBytes;
   float* m_sh = reinterpret_cast<float*>(ones_smem + kTcOnesBytes);        // [2][128]
-  float* scale_sh = m_sh + 2 * kTcRows;                                    // e4m3: [stage][4 K scales, 4 V scales]
-  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2], conv_full[4], conv_free[4]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes + C::kScaleBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 18);
+  float* rowc_sh = m_sh + 2 * kTcRows;                                     // e4m3: [128] score constant of the row
+  float* l_sh = rowc_sh + kTcRows;                                         // e4m3: [2][128] the sets' row sums
+  float* scale_sh = l_sh + 2 * kTcRows;                                    // e4m3: [stage][4 c, 4 a, 4 1/v, 4 unused]
+  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2][4]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes + kTcRowBytes + C::kScaleBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 16);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -248,25 +275,21 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
   const uint32_t bar_sfree = bar_pv + 16, bar_m = bar_sfree + 16;
-  const uint32_t conv_full0 = bar_m + 16, conv_free0 = conv_full0 + 32;  // four of each (e4m3)
   for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads)
-    reinterpret_cast<uint32_t*>(ones_smem)[i] = kFp8 ? 0x3C003C00u : 0x3F803F80u;  // 1.0 as f16 / bf16 pairs
+    reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;  // 1.0 as bf16 pairs (not used with e4m3)
   fence_proxy_async();  // read by the tensor core through the async proxy
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full0 + 8 * s, 1);
-      mbar_init(empty0 + 8 * s, kFp8 ? 4 : 1);  // released by the PV MMAs' commit, or by the 4 converter warps
-    }
-    for (int k = 0; k < 4; ++k) {
-      mbar_init(conv_full0 + 8 * k, 4);  // an operand block converted (4 converter warps)
-      mbar_init(conv_free0 + 8 * k, 1);  // the PV MMAs that read it have completed
+      mbar_init(empty0 + 8 * s, 1);  // released by the PV MMAs' commit
     }
     for (int k = 0; k < 2; ++k) {
       mbar_init(bar_s + 8 * k, 1);
       mbar_init(bar_p + 8 * k, 4);   // one arrival per warp of the softmax set that owns the iteration
       mbar_init(bar_pv + 8 * k, 1);
       mbar_init(bar_sfree + 8 * k, 4);
-      mbar_init(bar_m + 8 * k, 4);
+#pragma unroll
+      for (int w = 0; w < 4; ++w) mbar_init(bar_m + 8 * (4 * k + w), 1);  // per warp: rows w*32.. of set k
     }
     *cta_err = 0;
     fence_mbar_init();
@@ -283,12 +306,11 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTmemO;  // S buffer k at tmem_s + 64 k
-  const uint32_t tmem_q = tmem_base + kTmemQ, tmem_p = tmem_base + kTmemP;  // P buffer k at tmem_p + 32 k
+  const uint32_t tmem_q = tmem_base + kTmemQ<kFp8>, tmem_p = tmem_base + kTmemP<kFp8>;  // P buffer k at tmem_p + 32 k
 
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
 
-  // The roles, as closures: the two variants dispatch them differently (the e4m3 one by warpgroup, each
-  // group first taking or giving up registers).
+  // The roles, as closures.
   // ---- Q: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of S = Q . K^T
   auto load_q = [&]() {
     if (warp < 4) {
@@ -296,22 +318,53 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       const bool valid = r < rows_total;
       const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
       const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
+      if constexpr (!kFp8) {
   #pragma unroll
-      for (int h = 0; h < D / 64; ++h) {  // 64 bf16 = 32 columns per store
-        uint32_t qv[32];
+        for (int h = 0; h < D / 64; ++h) {  // 64 bf16 = 32 columns per store
+          uint32_t qv[32];
   #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint4 v = valid ? src[h * 8 + ch] : make_uint4(0u, 0u, 0u, 0u);
-          qv[4 * ch] = v.x; qv[4 * ch + 1] = v.y; qv[4 * ch + 2] = v.z; qv[4 * ch + 3] = v.w;
-          if (kFp8) {  // the e4m3 variant multiplies in f16: bf16 pairs -> f16 pairs
-  #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const uint32_t w = qv[4 * ch + e];
-              qv[4 * ch + e] = pack2<true>(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-            }
+          for (int ch = 0; ch < 8; ++ch) {
+            const uint4 v = valid ? src[h * 8 + ch] : make_uint4(0u, 0u, 0u, 0u);
+            qv[4 * ch] = v.x; qv[4 * ch + 1] = v.y; qv[4 * ch + 2] = v.z; qv[4 * ch + 3] = v.w;
           }
+          tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32 * h, qv);
         }
-        tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32 * h, qv);
+      } else {
+        // e4m3 x e4m3 on the tensor core: the row is scaled by a power of two so that its largest
+        // magnitude lies in [128, 256) and written as hi + lo, both e4m3 (|q - hi - lo| <= 2^-8 |q| or
+        // 2^-17 of the row's largest magnitude); the power of two goes into the row's score constant.
+        uint32_t qw[D / 2];
+        uint32_t amax = 0u;  // bf16 magnitudes order like their bit patterns
+  #pragma unroll
+        for (int ch = 0; ch < D / 8; ++ch) {
+          const uint4 v = valid ? src[ch] : make_uint4(0u, 0u, 0u, 0u);
+          qw[4 * ch] = v.x; qw[4 * ch + 1] = v.y; qw[4 * ch + 2] = v.z; qw[4 * ch + 3] = v.w;
+  #pragma unroll
+          for (int e = 0; e < 4; ++e)
+            amax = max(amax, max((qw[4 * ch + e] << 16) & 0x7fff0000u, qw[4 * ch + e] & 0x7fff0000u));
+        }
+        const int ex = static_cast<int>(amax >> 23);                      // biased exponent of the largest magnitude
+        const int up = (ex == 0 || ex == 255) ? 0 : min(max(134 - ex, -100), 100);  // it times 2^up is in [128, 256)
+        const float mul = __uint_as_float(static_cast<uint32_t>(127 + up) << 23);
+        rowc_sh[tid] = p.scale * 1.4426950408889634f * __uint_as_float(static_cast<uint32_t>(127 - up) << 23);
+        uint32_t qh[32], ql[32];
+  #pragma unroll
+        for (int c4 = 0; c4 < D / 4; ++c4) {  // four elements -> one 32-bit column of each part
+          uint32_t h2[2], l2[2];
+  #pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const uint32_t w = qw[2 * c4 + e];
+            const float x0 = __uint_as_float(w << 16) * mul, x1 = __uint_as_float(w & 0xffff0000u) * mul;
+            h2[e] = f32x2_to_e4m3x2(x0, x1);
+            uint32_t back16 = e4m3x2_to_f16x2(h2[e]);  // what the tensor core will read for the high parts
+            const float2 back = __half22float2(*reinterpret_cast<__half2*>(&back16));
+            l2[e] = f32x2_to_e4m3x2(x0 - back.x, x1 - back.y);
+          }
+          qh[c4] = h2[0] | (h2[1] << 16);
+          ql[c4] = l2[0] | (l2[1] << 16);
+        }
+        tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16), qh);
+        tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32, ql);
       }
       tmem_wait_st();
     }
@@ -329,7 +382,10 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     bool bad = false;
     int pg = 0;
-    float ks = 0.f, vs = 0.f;  // e4m3: the page's dequantisation factors
+    // e4m3, per page: the score factor (K scale), log2 of the V scale and its reciprocal. The scales are
+    // positive by construction; the clamps keep an all-zero or negative entry from producing inf or NaN.
+    // (lanes past the last page keep finite values: a masked score times 0 would be NaN)
+    float sc_c = 1.f, sc_a = 0.f, sc_i = 1.f;
     for (int it = 0; it < u_iters; ++it) {
       const int s = it % kTcStages;
       if ((it & 7) == 0) {  // page ids of the next 8 iterations (32 pages), one per lane
@@ -338,8 +394,12 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
           const int v = table[page0 + it * kTcPagesPerIter + lane];
           pg = (v < 0 || v >= p.geom.num_pages) ? -1 : v;
           if (kFp8) {
-            ks = p.k_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g];
-            vs = p.v_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g];
+            const float ks = fabsf(p.k_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g]);
+            const float vs = fabsf(p.v_scale[static_cast<int64_t>(max(pg, 0)) * p.geom.num_kv_heads + g]);
+            const float vc = fminf(fmaxf(vs, 8.6736174e-19f), 1.1529215e18f);  // 2^-60 .. 2^60
+            sc_c = fminf(fmaxf(ks, 1e-30f), 1e30f);
+            sc_a = __log2f(vc);
+            sc_i = 1.f / vc;
           }
         }
       }
@@ -349,29 +409,25 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       if (!ok) { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); break; }
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       const uint32_t stage = ring + s * kTcStageBytes, bar = full0 + 8 * s;
-      if (kFp8) {  // this stage's scales, written by the lanes that hold its pages (seen through the full barrier)
+      if (kFp8) {  // this stage's page constants, written by the lanes that hold its pages (seen through the full barrier)
         if ((lane >> 2) == (it & 7)) {
-          scale_sh[s * 8 + (lane & 3)] = ks;
-          scale_sh[s * 8 + 4 + (lane & 3)] = vs;
+          scale_sh[s * 16 + (lane & 3)] = sc_c;
+          scale_sh[s * 16 + 4 + (lane & 3)] = sc_a;
+          scale_sh[s * 16 + 8 + (lane & 3)] = sc_i;
         }
         __syncwarp();
       }
-      mbar_expect_tx_if(leader, bar, n_here * 2 * (kFp8 ? C::kRawTileBytes : kTcTileBytes));
+      mbar_expect_tx_if(leader, bar, n_here * 2 * kTcTileBytes);
       // K: one copy per 128-byte line so that page j's 16 rows follow page j-1's in each line block
-      // (an e4m3 row is one line; raw V tiles follow the raw K block)
+      // (an e4m3 row is one line)
       auto load_page = [&](int j) {
         const int page_raw = __shfl_sync(0xffffffffu, pg, (it & 7) * kTcPagesPerIter + j);
         bad |= page_raw < 0;
         const int page = max(page_raw, 0);
-        if (kFp8) {
-          tma_load_5d_if(leader, stage + j * C::kRawTileBytes, &k_map, bar, 0, g, page);
-          tma_load_5d_if(leader, stage + (kTcPagesPerIter + j) * C::kRawTileBytes, &v_map, bar, 0, g, page);
-        } else {
 #pragma unroll
-          for (int ln = 0; ln < C::kLines; ++ln)
-            tma_load_5d_if(leader, stage + ln * (kTcKBytes / C::kLines) + j * (kPageSize * 128), &k_map, bar, ln, g, page);
-          tma_load_5d_if(leader, stage + kTcKBytes + j * kTcTileBytes, &v_map, bar, 0, g, page);
-        }
+        for (int ln = 0; ln < C::kLines; ++ln)
+          tma_load_5d_if(leader, stage + ln * (kTcKBytes / C::kLines) + j * (kPageSize * 128), &k_map, bar, ln, g, page);
+        tma_load_5d_if(leader, stage + kTcKBytes + j * kTcTileBytes, &v_map, bar, 0, g, page);
       };
       if (n_here == kTcPagesPerIter) {
 #pragma unroll
@@ -396,150 +452,116 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     const int u_tail0 = __shfl_sync(0xffffffffu, L - page0 * kPageSize, 0);  // tokens from the first page to the end
     bool ok = true;
-    // the iteration's operand block: its ring stage (16-bit caches) or conversion slot (e4m3), and the
-    // phase parity of that block's "ready" barrier
-    constexpr uint32_t kBlocks = kFp8 ? C::kConvSlots : kTcStages;
-    const uint32_t blocks0 = kFp8 ? smem_u32(conv_smem) : ring;
-    const uint32_t ready0 = kFp8 ? conv_full0 : full0;
-    uint32_t stage_i = 0, stage_par = 0;
+    uint32_t stage_i = 0, stage_par = 0;  // the iteration's ring stage and the phase parity of its full barrier
     for (int it = 0; it < u_iters; ++it) {
       // S(it) overwrites the buffer of S(it-2): the softmax warps have loaded that into registers
       if (it >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (it & 1), ((it - 2) >> 1) & 1);
-      if (ok) ok = mbar_wait_bounded(ready0 + 8 * stage_i, stage_par);  // the block has landed / been converted
+      if (ok) ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);  // the block has landed
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      const uint32_t stage = blocks0 + stage_i * C::kOperandBytes;
+      const uint32_t stage = ring + stage_i * C::kOperandBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
       const int tail = u_tail0 - (it * kTcPagesPerIter + n_here - 1) * kPageSize;  // valid rows of the last page here
-      if (!kFp8 && tail < kPageSize) {  // clear the rows past the sequence end in V (P is 0 there, V must be
-                                        // finite); the e4m3 converters do it as they write the block
+      // P is 0 past the sequence end, but V must be finite there: clear those rows of the last page, and
+      // (e4m3, where an MMA step spans two pages) the missing second page of the last step
+      const bool odd = kFp8 && (n_here & 1);
+      if (tail < kPageSize || odd) {
         const uint32_t vt = stage + kTcKBytes + (n_here - 1) * kTcTileBytes;
-        constexpr int kChunksPerRow = D / 8;  // 16-byte chunks of a row
-        for (int i = lane; i < (kPageSize - tail) * kChunksPerRow; i += 32) {
-          const int r = tail + i / kChunksPerRow, ch = i % kChunksPerRow;
-          asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_off(r, ch)), "r"(0));
+        if constexpr (kFp8) {  // a row is one 128-byte line: the rows to clear are contiguous
+          const int first = max(min(tail, kPageSize), 0) * 128, end = (odd ? 2 : 1) * kTcTileBytes;
+          for (int i = first + lane * 16; i < end; i += 32 * 16)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + i), "r"(0));
+        } else {
+          constexpr int kChunksPerRow = D / 8;  // 16-byte chunks of a row
+          for (int i = lane; i < (kPageSize - tail) * kChunksPerRow; i += 32) {
+            const int r = tail + i / kChunksPerRow, ch = i % kChunksPerRow;
+            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(vt + tile_off(r, ch)), "r"(0));
+          }
         }
         fence_proxy_async();
         __syncwarp();
       }
       tc_fence_after();
       const uint32_t d = u_tmem + 64 * (it & 1);
-      // S[:, 0..64) = Q . K^T over the 64 stacked token rows, contraction over d in 8 steps of 16
+      // S[:, 0..64) = Q . K^T over the 64 stacked token rows
       // (rows of pages that were not loaded hold stale data: those columns are masked later)
       const uint64_t kd0 = tc_desc(stage, 16, 1024);
+      if constexpr (kFp8) {
+        // contraction over d in 4 steps of 32, once with the high and once with the low parts of Q;
+        // descriptor start addresses are in 16-byte units: +2 per k-step of 32 bytes
 #pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) {
-        // descriptor start addresses are in 16-byte units: +2 per k-step, next line block further on
-        const uint64_t bd = kd0 + static_cast<uint64_t>((ks >> 2) * (kTcKBytes / C::kLines / 16) + (ks & 3) * 2);
-        tc_mma_ts_if(leader, d, u_tmem + kTmemQ + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
+        for (int part = 0; part < 2; ++part)
+#pragma unroll
+          for (int ks = 0; ks < D / 32; ++ks)
+            tc_mma_ts_if<true>(leader, d, u_tmem + kTmemQ<true> + 32 * part + 8 * ks, kd0 + static_cast<uint64_t>(ks * 2),
+                               idesc_s, (part | ks) ? 1u : 0u);
+      } else {
+        // contraction over d in steps of 16
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          // +2 per k-step, next line block further on
+          const uint64_t bd = kd0 + static_cast<uint64_t>((ks >> 2) * (kTcKBytes / C::kLines / 16) + (ks & 3) * 2);
+          tc_mma_ts_if<false>(leader, d, u_tmem + kTmemQ<false> + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
+        }
       }
       tc_commit_if(leader, bar_s + 8 * (it & 1));
-      if (++stage_i == kBlocks) { stage_i = 0; stage_par ^= 1; }
+      if (++stage_i == kTcStages) { stage_i = 0; stage_par ^= 1; }
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   };
   auto pv_issue_role = [&]() {
     // ================= PV issue: O += P . V and l += P . 1 =================
     constexpr uint32_t idesc_pv = tc_idesc(D, true, kFp8);
-    constexpr uint32_t idesc_l = tc_idesc(16, false, kFp8);
+    constexpr uint32_t idesc_l = tc_idesc(16, false, false);
     const uint64_t ones_desc = tc_desc(smem_u32(ones_smem), 16, 1024);
     const uint32_t leader = elect_one();
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
     const int u_iters = __shfl_sync(0xffffffffu, n_iters, 0);
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     bool ok = true;
-    constexpr uint32_t kBlocks = kFp8 ? C::kConvSlots : kTcStages;
-    const uint32_t blocks0 = kFp8 ? smem_u32(conv_smem) : ring;
-    uint32_t stage_i = 0;  // the iteration's operand block: ring stage or conversion slot
+    uint32_t stage_i = 0;  // the iteration's ring stage
     for (int it = 0; it < u_iters; ++it) {
       ok = mbar_wait_bounded(bar_p + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t stage = blocks0 + stage_i * C::kOperandBytes;
+      const uint32_t stage = ring + stage_i * C::kOperandBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
-      // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page, V read MN-major
-      const uint32_t pa0 = u_tmem + kTmemP + 32 * (it & 1);
-      const uint64_t vd0 = tc_desc(stage + kTcKBytes, kPageSize * 128, 1024);  // LBO: next 64 columns of d, SBO: next 8 tokens
-      // and l += P[:, 16j .. 16j+16) . 1 : the row sums of exactly the P that multiplies V
-      auto pv_page = [&](int j) {
-        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-        tc_mma_ts_if(leader, u_tmem + kTmemO, pa0 + 8 * j, vd0 + static_cast<uint64_t>(j * (kTcTileBytes / 16)), idesc_pv, acc);
-        tc_mma_ts_if(leader, u_tmem + kTmemL, pa0 + 8 * j, ones_desc, idesc_l, acc);
-      };
-      if (n_here == kTcPagesPerIter) {
+      const uint32_t pa0 = u_tmem + kTmemP<kFp8> + 32 * (it & 1);
+      // V read MN-major. LBO: next 64 columns of d (bf16; an e4m3 line holds all 128), SBO: next 8 tokens
+      const uint64_t vd0 = tc_desc(stage + kTcKBytes, kPageSize * 128, 1024);
+      if constexpr (kFp8) {
+        // O[it % 2] += P[:, 32j .. 32j+32) . V : one K = 32 step per two pages (their tiles are contiguous),
+        // once with the high and once with the low parts of P; the row sums are kept by the softmax warps
+        auto pv_pair = [&](int j) {
 #pragma unroll
-        for (int j = 0; j < kTcPagesPerIter; ++j) pv_page(j);
+          for (int part = 0; part < 2; ++part)
+            tc_mma_ts_if<true>(leader, u_tmem + kTmemO + D * (it & 1), pa0 + 16 * part + 8 * j,
+                               vd0 + static_cast<uint64_t>(j * (2 * kTcTileBytes / 16)), idesc_pv,
+                               (it > 1 || j > 0 || part > 0) ? 1u : 0u);
+        };
+        pv_pair(0);
+        if (n_here > 2) pv_pair(1);
       } else {
-        for (int j = 0; j < n_here; ++j) pv_page(j);
+        // O += P[:, 16j .. 16j+16) . V_j : one K = 16 step per page
+        // and l += P[:, 16j .. 16j+16) . 1 : the row sums of exactly the P that multiplies V
+        auto pv_page = [&](int j) {
+          const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+          tc_mma_ts_if<false>(leader, u_tmem + kTmemO, pa0 + 8 * j, vd0 + static_cast<uint64_t>(j * (kTcTileBytes / 16)), idesc_pv, acc);
+          tc_mma_ts_if<false>(leader, u_tmem + kTmemL, pa0 + 8 * j, ones_desc, idesc_l, acc);
+        };
+        if (n_here == kTcPagesPerIter) {
+#pragma unroll
+          for (int j = 0; j < kTcPagesPerIter; ++j) pv_page(j);
+        } else {
+          for (int j = 0; j < n_here; ++j) pv_page(j);
+        }
       }
-      // the stage may be refilled (the conversion slot rewritten) once these MMAs have read it
-      tc_commit_if(leader, (kFp8 ? conv_free0 : empty0) + 8 * stage_i);
-      tc_commit_if(leader, bar_pv + 8 * (it & 1));    // O and l updated, P buffer free again
-      if (++stage_i == kBlocks) stage_i = 0;
+      tc_commit_if(leader, empty0 + 8 * stage_i);     // the stage may be refilled once these MMAs have read it
+      tc_commit_if(leader, bar_pv + 8 * (it & 1));    // O (and l) updated, P buffer free again
+      if (++stage_i == kTcStages) stage_i = 0;
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
-  };
-  auto convert_role = [&]() {
-    if constexpr (kFp8) {
-      // ================= e4m3 -> f16 converters: raw stage -> operand block in a conversion slot ==========
-      // cvt.rn.f16x2.e4m3x2 is exact, the page's scale is folded in (one f16 multiply), rows past the
-      // sequence end become zeros. A thread moves 4 K and 4 V chunks of 16 bytes per iteration (one of each
-      // per page): raw row, chunk c (swizzled by the row) -> 16-bit row, chunks 2 (c % 4), 2 (c % 4) + 1 of
-      // line c / 4.
-      const int ct = tid - kTcSoftmaxWarps * 32;  // 0..127
-      const uint32_t conv0 = smem_u32(conv_smem);
-      // This thread's four chunks never change: chunk q of its four is row r = 16 q + ct / 8 (page q of the
-      // iteration, slot ct / 8), raw chunk c = ct % 8. Offsets inside a raw half-stage / an operand block:
-      const int rr = ct >> 3, c = ct & 7, sw = rr & 7;
-      const uint32_t src_off = static_cast<uint32_t>(rr * 128 + ((c ^ sw) << 4));          // + q * raw tile
-      const int line = c >> 2, c2 = (c & 3) * 2;
-      const uint32_t k_off = static_cast<uint32_t>(line * (64 * 128) + rr * 128);           // + q * 16 rows
-      const uint32_t v_off = static_cast<uint32_t>(kTcKBytes + line * (kPageSize * 128) + rr * 128);  // + q * V tile
-      const uint32_t ch0 = static_cast<uint32_t>((c2 ^ sw) << 4), ch1 = static_cast<uint32_t>(((c2 + 1) ^ sw) << 4);
-      uint32_t slot = 0, slot_par = 0, stage_i = 0, stage_par = 0;
-      bool ok = true;
-      for (int it = 0; it < n_iters; ++it) {
-        ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);                        // raw tiles have landed
-        if (ok && it >= C::kConvSlots) ok = mbar_wait_bounded(conv_free0 + 8 * slot, slot_par ^ 1);  // PV(it - kConvSlots) done
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        const uint32_t raw = ring + stage_i * kTcStageBytes;
-        const uint32_t dst = conv0 + slot * C::kOperandBytes;
-        const float* sc = scale_sh + stage_i * 8;
-        const int n_here = min(kTcPagesPerIter, n_pages - it * kTcPagesPerIter);
-        const int valid_rows = min(L - (page0 + it * kTcPagesPerIter) * kPageSize, n_here * kPageSize);  // token rows of this block
-#pragma unroll
-        for (int q = 0; q < kTcPagesPerIter; ++q) {
-          if (q < n_here) {  // (uniform)
-            uint4 kin, vin, klo, khi, vlo, vhi;
-            const uint32_t src = raw + q * C::kRawTileBytes + src_off;
-            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kin.x), "=r"(kin.y), "=r"(kin.z), "=r"(kin.w) : "r"(src));
-            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(vin.x), "=r"(vin.y), "=r"(vin.z), "=r"(vin.w)
-                         : "r"(src + kTcPagesPerIter * C::kRawTileBytes));
-            e4m3x16_to_f16(kin, pack2<true>(sc[q], sc[q]), klo, khi);
-            e4m3x16_to_f16(vin, pack2<true>(sc[4 + q], sc[4 + q]), vlo, vhi);
-            if (q * kPageSize + rr >= valid_rows) {  // a row past the end of the sequence (last block only)
-              klo = make_uint4(0u, 0u, 0u, 0u); khi = klo; vlo = klo; vhi = klo;
-            }
-            const uint32_t kd = dst + k_off + q * (kPageSize * 128), vd = dst + v_off + q * kTcTileBytes;
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(kd + ch0), "r"(klo.x), "r"(klo.y), "r"(klo.z), "r"(klo.w));
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(kd + ch1), "r"(khi.x), "r"(khi.y), "r"(khi.z), "r"(khi.w));
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(vd + ch0), "r"(vlo.x), "r"(vlo.y), "r"(vlo.z), "r"(vlo.w));
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(vd + ch1), "r"(vhi.x), "r"(vhi.y), "r"(vhi.z), "r"(vhi.w));
-          }
-        }
-        fence_proxy_async();   // the tensor core reads the block through the async proxy
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive_tc(conv_full0 + 8 * slot);   // block ready for S and PV
-          mbar_arrive_tc(empty0 + 8 * stage_i);    // raw stage may be refilled
-        }
-        if (++slot == C::kConvSlots) { slot = 0; slot_par ^= 1; }
-        if (++stage_i == kTcStages) { stage_i = 0; stage_par ^= 1; }
-      }
-      if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
-    }
   };
   auto softmax_role = [&]() {
     // ================= softmax: TMEM lane t <-> query row t; set x takes iterations x, x+2, ... ==========
@@ -552,8 +574,15 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;  // this warp's TMEM lanes
     const float scale_log2 = p.scale * 1.4426950408889634f;
     const uint32_t my_s = bar_s + 8 * set, my_p = bar_p + 8 * set, my_pv = bar_pv + 8 * set;
-    const uint32_t my_sfree = bar_sfree + 8 * set, my_m = bar_m + 8 * set, other_m = bar_m + 8 * (set ^ 1);
-    float m_ref = -INFINITY;   // reference max the accumulated O and l (both in tensor memory) are scaled by
+    const uint32_t my_sfree = bar_sfree + 8 * set;
+    // the running maximum passes between the two warps that own the same 32 rows (same scheduler)
+    const uint32_t my_m = bar_m + 8 * (4 * set + (warp & 3)), other_m = bar_m + 8 * (4 * (set ^ 1) + (warp & 3));
+    float m_ref = -INFINITY;   // reference max the accumulated O and l are scaled by
+    // e4m3: this set's share of the row sum l (kept here, not in tensor memory) and the reference it is
+    // scaled by; the row's score constant (softmax scale, log2 e and the power of two Q was scaled by)
+    float l_set = 0.f, m_l = -INFINITY, rowc = 0.f;
+    if constexpr (kFp8) rowc = rowc_sh[t];
+    uint32_t sc_stage = set % kTcStages;  // ring stage of this set's next iteration
     bool alive = true;
     auto fail = [&]() { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; };
     for (int it = set; it < n_iters; it += 2) {
@@ -580,13 +609,45 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       // row maximum of the raw scores (the scale is positive), four independent chains
       float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      float mx;
+      // e4m3, per page j of the iteration: x = s cq[j] + aq[j] with cq = K scale x row constant and aq = log2
+      // of the V scale, i.e. the softmax runs on the scores plus log2(V scale): P then carries the V scale
+      // into P . V (V is multiplied as raw e4m3), and dividing the page's sum of P by the V scale (iq)
+      // gives its share of l.
+      float cq[4], aq[4], iq[4];
+      if constexpr (kFp8) {
+        // (written by the producer before the tiles' full barrier completed, which the S issue warp
+        // observed before the MMAs whose commit this warp has waited for)
+        const float4 c4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16);
+        const float4 a4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16 + 4);
+        const float4 i4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16 + 8);
+        cq[0] = c4.x * rowc; cq[1] = c4.y * rowc; cq[2] = c4.z * rowc; cq[3] = c4.w * rowc;
+        aq[0] = a4.x; aq[1] = a4.y; aq[2] = a4.z; aq[3] = a4.w;
+        iq[0] = i4.x; iq[1] = i4.y; iq[2] = i4.z; iq[3] = i4.w;
+        sc_stage += 2;
+        if (sc_stage >= kTcStages) sc_stage -= kTcStages;
+        float mxb[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // two chains per page
 #pragma unroll
-      for (int h = 0; h < 2; ++h)
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int j = 0; j < 32; ++j) mxs[j & 3] = fmaxf(mxs[j & 3], __uint_as_float(sv[h][j]));
-      const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * scale_log2;
-      // the reference after iteration it-1 comes from the other set
-      if (it > 0) {
+          for (int j = 0; j < 32; j += 4) {
+            const int q = h * 2 + (j >> 4);
+            mxs[q] = max3(mxs[q], __uint_as_float(sv[h][j]), __uint_as_float(sv[h][j + 1]));
+            mxb[q] = max3(mxb[q], __uint_as_float(sv[h][j + 2]), __uint_as_float(sv[h][j + 3]));
+          }
+        mx = fmaxf(fmaxf(fmaf(fmaxf(mxs[0], mxb[0]), cq[0], aq[0]), fmaf(fmaxf(mxs[1], mxb[1]), cq[1], aq[1])),
+                   fmaxf(fmaf(fmaxf(mxs[2], mxb[2]), cq[2], aq[2]), fmaf(fmaxf(mxs[3], mxb[3]), cq[3], aq[3])));
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int j = 0; j < 32; j += 2)
+            mxs[(j >> 1) & 3] = max3(mxs[(j >> 1) & 3], __uint_as_float(sv[h][j]), __uint_as_float(sv[h][j + 1]));
+        mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * scale_log2;
+      }
+      // bf16: the reference after iteration it-1 comes from the other set (one O for both). e4m3: each
+      // set runs an online softmax of its own over its iterations, with its own O.
+      if (!kFp8 && it > 0) {
         ok = mbar_spin_bounded(other_m, ((it - 1) >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
@@ -596,46 +657,84 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       float m_new = m_ref;
       if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = fmaxf(m_ref, mx);
       const bool need = m_new != m_ref && m_ref != -INFINITY;
-      m_sh[(it & 1) * kTcRows + t] = m_new;
-      __syncwarp();
-      if (lane == 0) mbar_arrive_tc(my_m);  // (release: the other set reads m_sh after its wait)
-      if (it >= 2) {  // PV(it-2) has finished reading the P buffer this iteration writes
-        ok = mbar_spin_bounded(my_pv, (k - 1) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) { fail(); break; }
+      if constexpr (!kFp8) {
+        m_sh[(it & 1) * kTcRows + t] = m_new;
+        __syncwarp();
+        if (lane == 0) mbar_arrive_tc(my_m);  // (release: the other set reads m_sh after its wait)
       }
-      if (it > 0 && __any_sync(0xffffffffu, need)) {
-        // O and l may only be touched once PV(it-1) has completed; PV(it) is not issued before this
-        // warp arrives on bar_p below, and the other set rescales only after PV(it)
-        ok = mbar_spin_bounded(bar_pv + 8 * (set ^ 1), ((it - 1) >> 1) & 1);
+      if (it > (kFp8 ? 1 : 0) && __any_sync(0xffffffffu, need)) {
+        // O and l may only be touched once the last PV into them has completed: PV(it-1), or (e4m3)
+        // this set's PV(it-2). PV(it) is not issued before this warp arrives on bar_p below, and (bf16)
+        // the other set rescales only after PV(it)
+        ok = kFp8 ? mbar_spin_bounded(my_pv, (k - 1) & 1)
+                  : mbar_spin_bounded(bar_pv + 8 * (set ^ 1), ((it - 1) >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
         tc_fence_after();
         const float alpha = need ? ex2(m_ref - m_new) : 1.f;
+        const uint32_t my_o = tmem_o + (kFp8 ? D * set : 0) + lane_base;
 #pragma unroll
-        for (int cb = 0; cb < D / 32 + 1; ++cb) {  // O, then the block of columns that holds l
+        for (int cb = 0; cb < D / 32 + (kFp8 ? 0 : 1); ++cb) {  // O, then (bf16) the block of columns that holds l
           uint32_t ov[32];
-          tmem_ld32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
+          tmem_ld32(my_o + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
-          tmem_st32(tmem_o + lane_base + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
+          tmem_st32(my_o + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
         }
         tmem_wait_st();
       }
       m_ref = m_new;
       const float ref = m_ref == -INFINITY ? 0.f : m_ref;
-      // P = exp2(S * scale_log2 - ref) as bf16 pairs into TMEM lane t: the A operand of O += P . V
-      // (one packed FMA per two elements; masked columns stay -inf -> 0)
-      const uint64_t c2 = f32x2(__float_as_uint(scale_log2), __float_as_uint(scale_log2));
-      const uint64_t nr2 = f32x2(__float_as_uint(-ref), __float_as_uint(-ref));
       uint32_t pw[32];
+      if constexpr (kFp8) {
+        if (m_l != m_ref) {  // this set's row sum follows the reference (changed here or by the other set)
+          l_set *= ex2(m_l - m_ref);
+          m_l = m_ref;
+        }
+        // P = exp2(x - ref) as hi + lo, both e4m3, four tokens to a column: columns 0..15 the high
+        // parts, 16..31 the low parts (the A operands of the two P . V products)
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const uint64_t x2 = fma_f32x2(f32x2(sv[j >> 4][(2 * j) & 31], sv[j >> 4][(2 * j + 1) & 31]), c2, nr2);
-        float x0, x1;
-        f32x2_split(x2, x0, x1);
-        pw[j] = pack2<kFp8>(ex2(x0), ex2(x1));  // (f16 pairs in the e4m3 variant, bf16 otherwise)
+        for (int q = 0; q < 4; ++q) {
+          const uint64_t c2 = f32x2(__float_as_uint(cq[q]), __float_as_uint(cq[q]));
+          const uint64_t nr2 = f32x2(__float_as_uint(aq[q] - ref), __float_as_uint(aq[q] - ref));
+          uint64_t sum2 = 0ull;
+#pragma unroll
+          for (int j = 8 * q; j < 8 * q + 8; j += 2) {  // two pairs = four tokens = one column
+            uint32_t hi[2], lo[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const uint64_t x2 = fma_f32x2(f32x2(sv[j >> 4][(2 * (j + e)) & 31], sv[j >> 4][(2 * (j + e) + 1) & 31]), c2, nr2);
+              float x0, x1;
+              f32x2_split(x2, x0, x1);
+              const float p0 = ex2(x0), p1 = ex2(x1);
+              sum2 = add_f32x2(sum2, f32x2(__float_as_uint(p0), __float_as_uint(p1)));
+              split_e4m3x2(p0, p1, hi[e], lo[e]);
+            }
+            pw[j >> 1] = hi[0] | (hi[1] << 16);
+            pw[16 + (j >> 1)] = lo[0] | (lo[1] << 16);
+          }
+          float s0, s1;
+          f32x2_split(sum2, s0, s1);
+          l_set = fmaf(s0 + s1, iq[q], l_set);
+        }
+      } else {
+        // P = exp2(S * scale_log2 - ref) as bf16 pairs into TMEM lane t: the A operand of O += P . V
+        // (one packed FMA per two elements; masked columns stay -inf -> 0)
+        const uint64_t c2 = f32x2(__float_as_uint(scale_log2), __float_as_uint(scale_log2));
+        const uint64_t nr2 = f32x2(__float_as_uint(-ref), __float_as_uint(-ref));
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const uint64_t x2 = fma_f32x2(f32x2(sv[j >> 4][(2 * j) & 31], sv[j >> 4][(2 * j + 1) & 31]), c2, nr2);
+          float x0, x1;
+          f32x2_split(x2, x0, x1);
+          pw[j] = pack2<false>(ex2(x0), ex2(x1));
+        }
+      }
+      if (it >= 2) {  // PV(it-2) has finished reading the P buffer this iteration writes
+        ok = mbar_spin_bounded(my_pv, (k - 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { fail(); break; }
       }
       tmem_st32(tmem_p + 32 * set + lane_base, pw);
       tmem_wait_st();
@@ -646,10 +745,22 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 
     // ---- finalise: the last iteration's reference (from the set that owned it) and the last PV
     bool ok = alive;
-    if (alive && n_iters > 0) {
+    if constexpr (kFp8) {
+      // this set's last PV, then its (reference, row sum) for the merge of the two accumulators
+      const int last = n_iters - 1 - ((n_iters - 1 - set) & 1);  // its last iteration, if any
+      if (alive && last >= set) {
+        ok = mbar_wait_bounded(my_pv, (last >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
+        tc_fence_after();
+      }
+      if (m_l != m_ref) l_set *= ex2(m_l - m_ref);
+      m_sh[set * kTcRows + t] = m_ref;
+      l_sh[set * kTcRows + t] = l_set;
+    } else if (alive && n_iters > 0) {
       const int last = n_iters - 1;
       if ((last & 1) != set) {
-        ok = mbar_spin_bounded(bar_m + 8 * (last & 1), (last >> 1) & 1);
+        ok = mbar_spin_bounded(bar_m + 8 * (4 * (last & 1) + (warp & 3)), (last >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) m_ref = m_sh[(last & 1) * kTcRows + t];
       }
@@ -665,13 +776,23 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int dev_err = max(err, *cta_err);
     if (dev_err && tid == 0) report(p.status, dev_err);
     const bool valid_row = r < rows_total;
-    const bool have = alive && ok && n_iters > 0;  // warp-uniform
+    bool have = alive && ok && n_iters > 0;  // warp-uniform
+    if constexpr (kFp8) have = have && *cta_err == 0;  // (the other set's view: its O is read below)
     float l = 0.f;
+    float w0 = 1.f, w1 = 0.f;  // e4m3: weights of the two sets' accumulators
     if (have) {
-      uint32_t lv[32];
-      tmem_ld32(tmem_base + kTmemL + lane_base, lv);
-      tmem_wait_ld();
-      l = __uint_as_float(lv[0]);
+      if constexpr (kFp8) {
+        const float m0 = m_sh[t], m1 = m_sh[kTcRows + t];
+        m_ref = fmaxf(m0, m1);
+        w0 = m0 == -INFINITY ? 0.f : ex2(m0 - m_ref);
+        w1 = m1 == -INFINITY ? 0.f : ex2(m1 - m_ref);
+        l = w0 * l_sh[t] + w1 * l_sh[kTcRows + t];
+      } else {
+        uint32_t lv[32];
+        tmem_ld32(tmem_base + kTmemL + lane_base, lv);
+        tmem_wait_ld();
+        l = __uint_as_float(lv[0]);
+      }
     }
     const bool live = !dev_err && have && l > 0.f;
     const float inv = live ? 1.f / l : 0.f;
@@ -684,6 +805,17 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       if (have) {
         tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
         tmem_wait_ld();
+        if constexpr (kFp8) {  // O = w0 O[0] + w1 O[1] (the second exists from two iterations on)
+#pragma unroll
+          for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * w0);
+          if (n_iters > 1) {
+            uint32_t o1[32];
+            tmem_ld32(tmem_o + D + lane_base + 32 * cb, o1);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(fmaf(__uint_as_float(o1[j]), w1, __uint_as_float(ov[j])));
+          }
+        }
       } else {
 #pragma unroll
         for (int j = 0; j < 32; ++j) ov[j] = 0u;
@@ -719,17 +851,13 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     else if (warp == kTcPvWarp) pv_issue_role();
     else if (warp < kTcSoftmaxWarps) softmax_role();
   } else {
-    // four warpgroups; registers go from the converter and control warps to the softmax warps (each group
-    // executes its setmaxnreg at the head of the code that only it runs)
+    // by warpgroup, each first taking or giving up registers (the setmaxnreg sits at the head of the code
+    // that only that group runs)
     if (warp < kTcSoftmaxWarps) {
       reg_alloc_inc<kTcRegsSoftmax>();
       load_q();
       wait_q();
       softmax_role();
-    } else if (warp < kTcSoftmaxWarps + 4) {
-      reg_alloc_dec<kTcRegsConvert>();
-      wait_q();
-      convert_role();
     } else {
       reg_alloc_dec<kTcRegsControl>();
       if (warp == kTcProducerWarp) {
@@ -741,7 +869,6 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
     }
   }
-
 
   // ---- teardown: everyone is done with tensor memory before it is released
   tc_fence_before();
