@@ -135,10 +135,11 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lbo_byt
          (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) |
          (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: f32 accumulate, A K-major, M = 128; A and B both bf16 (kind::f16, format 1) or
-// both e4m3 (kind::f8f6f4, format 0).
-__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major, bool e4m3) {
-  return (1u << 4) | ((e4m3 ? 0u : 1u) << 7) | ((e4m3 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+// Instruction descriptor: f32 accumulate, A K-major, M = 128. Operand formats: kind::f16 1 = bf16;
+// kind::f8f6f4 0 = e4m3, 1 = e5m2.
+constexpr uint32_t kFmtBf16 = 1, kFmtE4m3 = 0, kFmtE5m2 = 1;
+__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major, uint32_t a_fmt, uint32_t b_fmt) {
+  return (1u << 4) | (a_fmt << 7) | (b_fmt << 10) | ((b_mn_major ? 1u : 0u) << 16) |
          (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTcRows >> 4) << 24);
 }
 template <uint32_t kRegs>
@@ -156,13 +157,20 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
   asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
   return r;
 }
-// x = hi + lo with both parts e4m3: hi keeps the top three mantissa bits of x (exact in e4m3 from 2^-6
-// up), lo is the remainder rounded. |x - hi - lo| <= max(2^-7 |x|, 2^-10); 0 <= x <= 448 or so.
-__device__ __forceinline__ void split_e4m3x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
-  const float t0 = __uint_as_float(__float_as_uint(x0) & 0xfff00000u);
-  const float t1 = __uint_as_float(__float_as_uint(x1) & 0xfff00000u);
-  hi = f32x2_to_e4m3x2(t0, t1);
-  lo = f32x2_to_e4m3x2(x0 - t0, x1 - t1);
+// x = hi + lo, hi in e4m3 (x rounded to nearest), lo in e5m2 (the remainder, rounded): two bytes of each
+// for two values, 0 <= x <= 448. |x - hi - lo| <= max(2^-7 |x|, 2^-17): the wider exponent range of e5m2
+// keeps the weights far below the row's largest one (e4m3 alone stops at 2^-9) to three significant bits.
+// The remainder is taken in f16 pairs, where it is exact.
+__device__ __forceinline__ void split_e4m3_e5m2_x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  uint32_t xh, back;
+  uint16_t h, l;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(xh) : "f"(x1), "f"(x0));
+  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(h) : "r"(xh));
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(h));
+  asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(xh) : "r"(xh), "r"(back));
+  asm("cvt.rn.satfinite.e5m2x2.f16x2 %0, %1;" : "=h"(l) : "r"(xh));
+  hi = h;
+  lo = l;
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -444,7 +452,8 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     // instructions of both per iteration at one every 4-8 clocks, which is as long as the iteration
     // itself. Each keeps to its own chain of barriers; the tensor core's order between the two does not
     // matter.)
-    constexpr uint32_t idesc_s = tc_idesc(kTcPagesPerIter * kPageSize, false, kFp8);
+    constexpr uint32_t idesc_s = kFp8 ? tc_idesc(kTcPagesPerIter * kPageSize, false, kFmtE4m3, kFmtE4m3)
+                                      : tc_idesc(kTcPagesPerIter * kPageSize, false, kFmtBf16, kFmtBf16);
     const uint32_t leader = elect_one();
     // warp-uniform copies (a shuffle from lane 0 tells the compiler so)
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
@@ -511,8 +520,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   };
   auto pv_issue_role = [&]() {
     // ================= PV issue: O += P . V and l += P . 1 =================
-    constexpr uint32_t idesc_pv = tc_idesc(D, true, kFp8);
-    constexpr uint32_t idesc_l = tc_idesc(16, false, false);
+    constexpr uint32_t idesc_pv = kFp8 ? tc_idesc(D, true, kFmtE4m3, kFmtE4m3) : tc_idesc(D, true, kFmtBf16, kFmtBf16);
+    constexpr uint32_t idesc_pv_lo = tc_idesc(D, true, kFmtE5m2, kFmtE4m3);  // e4m3 caches: the low parts of P are e5m2
+    constexpr uint32_t idesc_l = tc_idesc(16, false, kFmtBf16, kFmtBf16);
     const uint64_t ones_desc = tc_desc(smem_u32(ones_smem), 16, 1024);
     const uint32_t leader = elect_one();
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
@@ -537,7 +547,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
           for (int part = 0; part < 2; ++part)
             tc_mma_ts_if<true>(leader, u_tmem + kTmemO + D * (it & 1), pa0 + 16 * part + 8 * j,
-                               vd0 + static_cast<uint64_t>(j * (2 * kTcTileBytes / 16)), idesc_pv,
+                               vd0 + static_cast<uint64_t>(j * (2 * kTcTileBytes / 16)), part ? idesc_pv_lo : idesc_pv,
                                (it > 1 || j > 0 || part > 0) ? 1u : 0u);
         };
         pv_pair(0);
@@ -692,7 +702,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
           l_set *= ex2(m_l - m_ref);
           m_l = m_ref;
         }
-        // P = exp2(x - ref) as hi + lo, both e4m3, four tokens to a column: columns 0..15 the high
+        // P = exp2(x - ref) as hi (e4m3) + lo (e5m2), four tokens to a column: columns 0..15 the high
         // parts, 16..31 the low parts (the A operands of the two P . V products)
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -709,7 +719,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
               f32x2_split(x2, x0, x1);
               const float p0 = ex2(x0), p1 = ex2(x1);
               sum2 = add_f32x2(sum2, f32x2(__float_as_uint(p0), __float_as_uint(p1)));
-              split_e4m3x2(p0, p1, hi[e], lo[e]);
+              split_e4m3_e5m2_x2(p0, p1, hi[e], lo[e]);
             }
             pw[j >> 1] = hi[0] | (hi[1] << 16);
             pw[16 + (j >> 1)] = lo[0] | (lo[1] << 16);

@@ -90,6 +90,54 @@ def test_verify_attention_fp8_and_causal_needle(oracle):
 
 
 @pytest.mark.parametrize("flags", MQ)
+@pytest.mark.parametrize("spread", ["moderate", "extreme"])
+def test_verify_fp8_under_unequal_scales(oracle, flags, spread):
+    """e4m3 caches whose page scales differ by powers of two (the tensor-core path folds the K scale into
+    the score factor and the V scale into the exponent and divides it out of the row sum), pages with a
+    zero scale, query rows of very different magnitude (Q is split into two e4m3 parts after a per-row
+    power-of-two scaling), and a lone dominant key (P = 1 next to tiny weights).
+    moderate: V scales within 2^-3 .. 2^3 of each other, checked with the element-wise tolerance.
+    extreme: V scales over 2^-12 .. 2^8, values in the hundreds: the weights P reach the tensor core as
+    e4m3 + e5m2 pairs (2^-7 relative), so the bound is relative to the row's largest output, 1 %."""
+    rng = np.random.default_rng(77)
+    lens = [1000, 333, 64, 17]
+    T = 8
+    w = W.make_workload("fp8_scales", lens, 32, 8, 128, kv_dtype="e4m3", seed=78)
+    used = np.unique(w.block_table[w.block_table >= 0])
+    ks, vs = w.k_scale.copy(), w.v_scale.copy()
+    vexp = (-3, 4) if spread == "moderate" else (-12, 9)
+    ks[used] *= np.exp2(rng.integers(-3, 2, size=ks[used].shape)).astype(np.float32)
+    vs[used] *= np.exp2(rng.integers(*vexp, size=vs[used].shape)).astype(np.float32)
+    vs[used[3]] = 0.0                                   # a page whose values all decode to zero
+    vs[used[10], 2] = 0.0
+    q = W.bf16_bits_to_f32(verify_inputs(w, T, 79)[0])
+    q *= np.exp2(rng.integers(-8, 3, size=q.shape[:3])).astype(np.float32)[..., None]   # per (b, t, head)
+    # a dominant key: row (b=0, t=T-1, head 5) points at the cache row of token 500 of sequence 0
+    page, slot, g = int(w.block_table[0, 500 // 16]), 500 % 16, 5 // 4
+    dec = np.asarray(oracle.e4m3_decode_table(), dtype=np.float64)
+    krow = (dec[w.k_cache[page, g, slot]] * float(ks[page, g])).astype(np.float32)
+    q[0, T - 1, 5] = (60.0 / (float(w.scale) * float(krow @ krow))) * krow
+    q = W.f32_to_bf16_bits(q.astype(np.float32))
+    ref, _ = oracle.paged_verify_attention(q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.scale, ks, vs)
+    dw = DeviceWorkload(w)
+    out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                     float(w.scale), k_scale=torch.from_numpy(ks).cuda(),
+                                     v_scale=torch.from_numpy(vs).cuda(), flags=flags, status=dw.status)
+    got = bf16_to_f64(out)
+    if spread == "moderate":
+        assert_close(got, ref, "e4m3", what=f"fp8 unequal scales flags {flags}")
+    else:
+        assert np.isfinite(got).all()
+        row_max = np.abs(ref).max(axis=-1, keepdims=True)
+        worst = (np.abs(got - ref) / (2e-2 + 1e-2 * row_max)).max()
+        assert worst <= 1.0, f"fp8 extreme scales flags {flags}: max err / (2e-2 + 1% of row max) = {worst:.3f}"
+    # the dominant key's row is that value row (times its scale), to the rounding of the output
+    vrow = dec[w.v_cache[page, g, slot]] * float(vs[page, g])
+    assert np.abs(got[0, T - 1, 5] - vrow).max() <= 2e-2 + 2e-2 * np.abs(vrow).max()
+    assert int(dw.status.item()) == 0
+
+
+@pytest.mark.parametrize("flags", MQ)
 @pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
 @pytest.mark.parametrize("B", [3, 40])
 def test_shared_prefix_cascade(oracle, kv_dtype, B, flags):
