@@ -1,7 +1,7 @@
 // Multi-query paged attention on the 5th-generation tensor cores (tcgen05 + TMEM): verification of a
 // block of draft tokens, and the shared-prefix part of a decode batch; same contract as attention_mq.cu.
 // Up to 128 query rows (query tokens x group size) per CTA against one sequence's pages. bf16 KV with
-// head_dim 128 or 64 (the figures in this comment are for 128), or e4m3 KV with head_dim 128.
+// head_dim 128 or 64 (the figures in this comment are for bf16 and 128), or e4m3 KV with head_dim 128.
 //
 // This is the part of the path that is a real dense contraction, so it runs as
 // UMMA tiles with operands and accumulators in tensor memory (TMEM, 128 lanes = query rows):
@@ -35,12 +35,20 @@
 //               TMEM when the max grew by more than 2^8 -> wait PV(i-2) (P buffer free) -> P =
 //               exp2(S * scale - ref) as bf16 pairs (packed f32x2 FMA, one exp2 per element) ->
 //               tcgen05.st P -> arrive(bar_p[i&1])
-// e4m3 KV: the tensor core has no bf16 x e4m3 mode and e4m3 x e4m3 would quantise Q and P, so the tiles
-// are converted. The TMA ring holds the raw tiles (128-byte rows), four converter warps (8-11) write
-// each iteration's K and V as an f16 operand block (exact conversion, the page's scale folded in, rows
-// past the sequence end zeroed) into one of three conversion slots, and Q, P and the tile of ones are
-// f16 as well. That variant runs 16 warps (producer 12, S issue 13, PV issue 14) as four warpgroups and
-// moves registers from the converter and control groups to the softmax groups (setmaxnreg).
+// e4m3 KV: the tensor core has no bf16 x e4m3 mode, so the products run as e4m3 x e4m3 (kind::f8f6f4,
+// K = 32) on the tiles as they lie in the cache, and Q and P are each written as two 8-bit parts, one
+// more MMA per part into the same accumulator:
+//   Q = hi + lo, both e4m3, after a per-row power of two that brings the row's largest magnitude into
+//       [128, 256) (it goes into the row's score constant): 2 x 4 MMAs M128 x N64 x K32 per iteration
+//   P = hi (e4m3, round to nearest) + lo (e5m2: its exponent range keeps weights far below the row's
+//       largest one, where e4m3 stops at 2^-9): 2 x 2 MMAs M128 x N128 x K32, a step spanning two pages
+//       whose V tiles are contiguous; |p - hi - lo| <= max(2^-7 p, 2^-17)
+// The page scales stay out of the tiles: the K scale is the score factor of the page's 16 columns; the V
+// scale enters as log2(v_scale) added to the score, so that P carries it into P . V_raw, and each page's
+// sum of P divided by v_scale is its share of the row sum, which the softmax warps keep in registers.
+// Each softmax set has an O of its own (and its own running maximum and row sum), merged at the end
+// like split-KV partials, so the sets exchange nothing per iteration. A twelfth, idle warp completes
+// the third warpgroup so that setmaxnreg can move registers from the control warps to the softmax warps.
 // All mbarrier waits are bounded; TMEM is always released before the CTA exits.
 #include "common.cuh"
 #include "tma_ptx.cuh"
@@ -80,12 +88,12 @@ constexpr int kTcSoftmaxWarps = 8;      // two sets of 4: set x takes the iterat
 // e4m3: three warpgroups start with 168 registers a thread; the control group keeps 72 and each softmax
 // group takes 208 (setmaxnreg): 2 x 128 x 208 + 128 x 72 <= 65536. With 168 the softmax loop spilled.
 constexpr uint32_t kTcRegsSoftmax = 208, kTcRegsControl = 72;
-// Tensor memory columns (32-bit each, 128 lanes = query rows): S buffers 0..63 and 64..127 (f32),
-// O 128..255 (f32), Q 256..319 (bf16 pairs along d; e4m3: the high parts in 256..287, four to a column,
-// the low parts in 288..319), P buffers 320..351 and 352..383 (bf16 pairs along tokens; e4m3: 16 columns
-// of high parts, then 16 of low parts). Allocations are powers of two.
-// e4m3: each softmax set accumulates into an O of its own (128..255 and 256..383; the two are merged at
-// the end like split-KV partials), Q 384..447, P buffers 448..479 and 480..511.
+// Tensor memory columns (32-bit each, 128 lanes = query rows), bf16: S buffers 0..63 and 64..127 (f32),
+// O 128..255 (f32), Q 256..319 (bf16 pairs along d), P buffers 320..351 and 352..383 (bf16 pairs along
+// tokens), l 384..399. Allocations are powers of two.
+// e4m3: S as above; each softmax set accumulates into an O of its own (128..255 and 256..383); Q 384..447
+// (four elements to a column: 32 columns of high parts, then 32 of low parts); P buffers 448..479 and
+// 480..511 (four tokens to a column: 16 columns of high parts, then 16 of low parts).
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemO = 128, kTmemL = 384;  // l (bf16): row sums of P, 16 columns (all equal)
 template <bool kFp8> constexpr uint32_t kTmemQ = kFp8 ? 384 : 256;
