@@ -203,6 +203,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 // Packed pairs of f32 (sm_100): one instruction per two elements in the softmax inner loops.
 __device__ __forceinline__ uint64_t f32x2(uint32_t lo, uint32_t hi) {
   uint64_t r;
@@ -245,6 +253,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes + kTcRowBytes + C::kScaleBytes);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 16);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
+  int* rank_slot = cta_err + 1;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.group, T = mp.n_q;
@@ -252,48 +261,31 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const int n_rb = (rows_total + kTcRows - 1) / kTcRows;
   const int c = blockIdx.x, g = blockIdx.y / n_rb, rb = blockIdx.y % n_rb;
   const bool split = p.chunk_tokens > 0;
+  // unsplit units differ in length: the CTA with blockIdx.z = r serves the r-th longest sequence
+  const bool ranked = !split && mp.kv_len_fixed == 0 && p.batch > 1 && p.batch <= 128;
   int b = blockIdx.z;
-  if (!split && mp.kv_len_fixed == 0 && p.batch > 1 && p.batch <= 128) {  // (ranking costs O(batch^2/threads))
-    // unsplit units differ in length: the CTA with blockIdx.z = r serves the r-th longest sequence
-    int* lens = reinterpret_cast<int*>(smem);
-    for (int j = tid; j < p.batch; j += kTcThreads) lens[j] = max(p.seq_lens[j], 0);
-    __syncthreads();
-    for (int j = tid; j < p.batch; j += kTcThreads) {
-      const int Lj = lens[j];
-      int rank = 0;
-      for (int i = 0; i < p.batch; ++i) rank += (lens[i] > Lj) || (lens[i] == Lj && i < j);
-      if (rank == static_cast<int>(blockIdx.z)) *cta_err = j;
-    }
-    __syncthreads();
-    b = *cta_err;
-    __syncthreads();  // lens aliases the ring and cta_err is reused below
-  }
-
-  const int L = mp.kv_len_fixed > 0 ? mp.kv_len_fixed : max(p.seq_lens[b], 0);
-  int t0 = p.first_token, t1 = L;
-  if (split) {
-    t0 = p.first_token + c * p.chunk_tokens;
-    if (t0 >= L) return;
-    t1 = min(t0 + p.chunk_tokens, L);
+  // Everything below up to the roles is the serial start of the CTA (about 5 us before the first P): the
+  // set-up that does not depend on the sequence comes first and shares its barrier with the ranking.
+  // (the loads of the status word and of the lengths are issued together: each is a trip to L2 or DRAM)
+  const int32_t status_now = p.status != nullptr ? *reinterpret_cast<volatile int32_t*>(p.status) : 0;
+  int len_mine = 0;  // ranked: the length of sequence tid
+  if (ranked && tid < p.batch) len_mine = max(p.seq_lens[tid], 0);
+  if (split) {  // an empty chunk leaves before anything is allocated
+    const int Lb = mp.kv_len_fixed > 0 ? mp.kv_len_fixed : max(p.seq_lens[b], 0);
+    if (p.first_token + c * p.chunk_tokens >= Lb) return;
   }
   // once any CTA of this launch has reported a timed-out wait, the rest do not start
-  if (p.status != nullptr && *reinterpret_cast<volatile int32_t*>(p.status) == PDA_DEV_TIMEOUT) return;
-  int err = 0;
-  if (static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
-      (split && static_cast<int64_t>(L - p.first_token) >
-                    static_cast<int64_t>(p.max_chunks - p.chunk_slot0) * p.chunk_tokens))
-    err = PDA_DEV_BAD_SEQ_LEN;
-  const int page0 = t0 / kPageSize;
-  const int n_pages = err ? 0 : (t1 + kPageSize - 1) / kPageSize - page0;
-  const int n_iters = (n_pages + kTcPagesPerIter - 1) / kTcPagesPerIter;
+  if (status_now == PDA_DEV_TIMEOUT) return;
 
   const uint32_t ring = smem_u32(smem);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
   const uint32_t bar_sfree = bar_pv + 16, bar_m = bar_sfree + 16;
-  for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads)
-    reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;  // 1.0 as bf16 pairs (not used with e4m3)
-  fence_proxy_async();  // read by the tensor core through the async proxy
+  if constexpr (!kFp8) {
+    for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads)
+      reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;  // 1.0 as bf16 pairs
+    fence_proxy_async();  // read by the tensor core through the async proxy
+  }
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full0 + 8 * s, 1);
@@ -316,10 +308,46 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
                  ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-
+  if (ranked) {
+    int* lens = reinterpret_cast<int*>(smem);  // (aliases the ring, which nothing writes before the barrier below)
+    if (tid < p.batch) lens[tid] = len_mine;  // (batch <= 128 < threads)
+    __syncthreads();
+    // rank of sequence j = how many come before it (longer, or as long with a lower index); `parts` lanes
+    // share a sequence's comparisons
+    int parts = 1;
+    while (parts < 32 && parts * 2 * p.batch <= kTcThreads) parts *= 2;
+    const int j = tid / parts, part = tid % parts;
+    int rank = 0;
+    if (j < p.batch) {
+      const int Lj = lens[j];
+      for (int i = part; i < p.batch; i += parts) rank += (lens[i] > Lj) || (lens[i] == Lj && i < j);
+    }
+    for (int o = 1; o < parts; o <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+    if (j < p.batch && part == 0 && rank == static_cast<int>(blockIdx.z)) {
+      rank_slot[0] = j;
+      rank_slot[1] = lens[j];
+    }
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (ranked) b = rank_slot[0];
+
+  const int L = mp.kv_len_fixed > 0 ? mp.kv_len_fixed : ranked ? rank_slot[1] : max(p.seq_lens[b], 0);
+  int t0 = p.first_token, t1 = L;
+  if (split) {
+    t0 = p.first_token + c * p.chunk_tokens;
+    t1 = min(t0 + p.chunk_tokens, L);
+  }
+  int err = 0;
+  if (static_cast<int64_t>(L) > static_cast<int64_t>(p.block_table_stride) * kPageSize ||
+      (split && static_cast<int64_t>(L - p.first_token) >
+                    static_cast<int64_t>(p.max_chunks - p.chunk_slot0) * p.chunk_tokens))
+    err = PDA_DEV_BAD_SEQ_LEN;
+  const int page0 = t0 / kPageSize;
+  const int n_pages = err ? 0 : (t1 + kPageSize - 1) / kPageSize - page0;
+  const int n_iters = (n_pages + kTcPagesPerIter - 1) / kTcPagesPerIter;
+
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTmemO;  // S buffer k at tmem_s + 64 k
   const uint32_t tmem_q = tmem_base + kTmemQ<kFp8>, tmem_p = tmem_base + kTmemP<kFp8>;  // P buffer k at tmem_p + 32 k
@@ -329,43 +357,46 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   // The roles, as closures.
   // ---- Q: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of S = Q . K^T
   auto load_q = [&]() {
-    if (warp < 4) {
-      const int r = rb * kTcRows + tid;
+    // the two softmax warps that own the same 32 rows (w and w + 4) take half a row each
+    if (warp < kTcSoftmaxWarps && (warp >> 2) < D / 64) {
+      const int t = tid & (kTcRows - 1), half = warp >> 2;
+      const int r = rb * kTcRows + t;
       const bool valid = r < rows_total;
       const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
       const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
+      const uint32_t my_q = tmem_q + (static_cast<uint32_t>((warp & 3) * 32) << 16);
       if constexpr (!kFp8) {
+        uint32_t qv[32];  // 64 bf16 = 32 columns
   #pragma unroll
-        for (int h = 0; h < D / 64; ++h) {  // 64 bf16 = 32 columns per store
-          uint32_t qv[32];
-  #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {
-            const uint4 v = valid ? src[h * 8 + ch] : make_uint4(0u, 0u, 0u, 0u);
-            qv[4 * ch] = v.x; qv[4 * ch + 1] = v.y; qv[4 * ch + 2] = v.z; qv[4 * ch + 3] = v.w;
-          }
-          tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32 * h, qv);
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint4 v = valid ? src[half * 8 + ch] : make_uint4(0u, 0u, 0u, 0u);
+          qv[4 * ch] = v.x; qv[4 * ch + 1] = v.y; qv[4 * ch + 2] = v.z; qv[4 * ch + 3] = v.w;
         }
+        tmem_st32(my_q + 32 * half, qv);
       } else {
         // e4m3 x e4m3 on the tensor core: the row is scaled by a power of two so that its largest
         // magnitude lies in [128, 256) and written as hi + lo, both e4m3 (|q - hi - lo| <= 2^-8 |q| or
         // 2^-17 of the row's largest magnitude); the power of two goes into the row's score constant.
-        uint32_t qw[D / 2];
+        // (Both warps read the whole row for the magnitude; each converts its half.)
+        uint32_t qw[D / 4];
         uint32_t amax = 0u;  // bf16 magnitudes order like their bit patterns
   #pragma unroll
         for (int ch = 0; ch < D / 8; ++ch) {
           const uint4 v = valid ? src[ch] : make_uint4(0u, 0u, 0u, 0u);
-          qw[4 * ch] = v.x; qw[4 * ch + 1] = v.y; qw[4 * ch + 2] = v.z; qw[4 * ch + 3] = v.w;
+          const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
   #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            amax = max(amax, max((qw[4 * ch + e] << 16) & 0x7fff0000u, qw[4 * ch + e] & 0x7fff0000u));
+          for (int e = 0; e < 4; ++e) {
+            amax = max(amax, max((w4[e] << 16) & 0x7fff0000u, w4[e] & 0x7fff0000u));
+            if ((ch >> 3) == half) qw[4 * (ch & 7) + e] = w4[e];
+          }
         }
         const int ex = static_cast<int>(amax >> 23);                      // biased exponent of the largest magnitude
         const int up = (ex == 0 || ex == 255) ? 0 : min(max(134 - ex, -100), 100);  // it times 2^up is in [128, 256)
         const float mul = __uint_as_float(static_cast<uint32_t>(127 + up) << 23);
-        rowc_sh[tid] = p.scale * 1.4426950408889634f * __uint_as_float(static_cast<uint32_t>(127 - up) << 23);
-        uint32_t qh[32], ql[32];
+        if (half == 0) rowc_sh[t] = p.scale * 1.4426950408889634f * __uint_as_float(static_cast<uint32_t>(127 - up) << 23);
+        uint32_t qh[16], ql[16];
   #pragma unroll
-        for (int c4 = 0; c4 < D / 4; ++c4) {  // four elements -> one 32-bit column of each part
+        for (int c4 = 0; c4 < D / 8; ++c4) {  // four elements -> one 32-bit column of each part
           uint32_t h2[2], l2[2];
   #pragma unroll
           for (int e = 0; e < 2; ++e) {
@@ -379,8 +410,8 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
           qh[c4] = h2[0] | (h2[1] << 16);
           ql[c4] = l2[0] | (l2[1] << 16);
         }
-        tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16), qh);
-        tmem_st32(tmem_q + (static_cast<uint32_t>(warp * 32) << 16) + 32, ql);
+        tmem_st16(my_q + 16 * half, qh);
+        tmem_st16(my_q + 32 + 16 * half, ql);
       }
       tmem_wait_st();
     }
