@@ -214,9 +214,16 @@ int kv_append_tokens_fp8(const void* k_new, const void* v_new, void* k_cache, vo
  *             inside this call.  `out` is always written.
  * The query rows of a kv head's group form dense tensor-core tiles (rows = tokens x
  * group size), so each page is fetched once per block, not once per token.
- * bf16 KV with head_dim 128 runs on tcgen05 tensor-core tiles with the accumulators
- * in tensor memory (128 query rows per CTA); other supported shapes (head_dim 64
- * bf16, 128 e4m3) and PDA_FLAG_MQ_MMA_SYNC use the mma.sync kernel. */
+ * bf16 KV with head_dim 128 or 64 and e4m3 KV with head_dim 128 run on tcgen05
+ * tensor-core tiles with the accumulators in tensor memory (128 query rows per CTA);
+ * PDA_FLAG_MQ_MMA_SYNC selects the mma.sync kernel instead.
+ * e4m3 on tcgen05: the products are e4m3 x e4m3 on the cache's bytes; q and the softmax
+ * weights enter as two 8-bit parts each (q to 2^-8, a weight to 2^-7 relative), the
+ * page scales through the softmax. An output element is within about 0.3 % of the
+ * largest magnitude in its row of the exact result, which meets 2e-2 + 2e-2 |ref| for
+ * values of order one; where the dequantised values are far larger, or a tighter
+ * bound is wanted, use PDA_FLAG_MQ_MMA_SYNC (weights in f16). Scales must be finite
+ * and non-negative (kv_append_fp8 writes them so). */
 int paged_verify_attention(const void* q, const void* k_cache, const void* v_cache,
                            const pda_cache_desc* desc, const float* k_scale,
                            const float* v_scale, const int32_t* block_table,
@@ -248,7 +255,9 @@ int paged_verify_attention(const void* q, const void* k_cache, const void* v_cac
  * also valid while `stream` is being captured; the side stream is created by the
  * first call that is not inside a capture, and until it exists the launches simply
  * follow one another on `stream`). Supported: group size <= 8, head_dim 64/128
- * (bf16) or 128 (e4m3), batch <= 4096. */
+ * (bf16) or 128 (e4m3), batch <= 4096. The prefix launch is a multi-query call:
+ * the kernel choice, `flags` and the e4m3 precision note of paged_verify_attention
+ * apply to it. */
 int paged_prefix_decode_attention(const void* q, const void* k_cache, const void* v_cache,
                                   const pda_cache_desc* desc, const float* k_scale,
                                   const float* v_scale, const int32_t* block_table,
