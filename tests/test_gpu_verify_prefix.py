@@ -89,6 +89,37 @@ def test_verify_attention_fp8_and_causal_needle(oracle):
     assert np.abs(out[0, :-1]).max() < 3.0    # N(0,1) averages, nowhere near 1..128
 
 
+@pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
+def test_verify_batch_beyond_the_ranked_range(oracle, kv_dtype):
+    """More than 128 sequences: the CTAs take the sequences in index order instead of longest first;
+    lengths from one token to a few pages, so that single-iteration CTAs and odd page counts occur."""
+    rng = np.random.default_rng(91)
+    B, T = 150, 3
+    lens = np.maximum(rng.integers(1, 200, size=B), T)
+    w = W.make_workload("big_batch", lens, 32, 8, 128, kv_dtype=kv_dtype, seed=92)
+    q, kn, vn = verify_inputs(w, T, 93)
+    dw = DeviceWorkload(w)
+    if kv_dtype == "bf16":  # (a bf16 workload's last slots are filled by the append)
+        k, v = w.k_cache.copy(), w.v_cache.copy()
+        oracle.kv_append_tokens(kn, vn, k, v, w.block_table, w.seq_lens)
+        pda.kv_append_tokens(bf16_tensor(kn), bf16_tensor(vn), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens)
+        ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
+    else:
+        ref, _ = oracle.paged_verify_attention(q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.scale,
+                                               w.k_scale, w.v_scale)
+    for chunk in (0, 64):
+        po = pl = None
+        if chunk:
+            mc = pda.max_chunks(int(lens.max()), chunk)
+            po = torch.full((B, T, 32, mc, 128), float("nan"), dtype=torch.float32, device="cuda")
+            pl = torch.full((B, T, 32, mc), float("nan"), dtype=torch.float32, device="cuda")
+        out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                         float(w.scale), chunk_tokens=chunk, part_o=po, part_lse=pl,
+                                         k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+        assert_close(bf16_to_f64(out), ref, kv_dtype, what=f"verify batch {B} {kv_dtype} chunk {chunk}")
+    assert int(dw.status.item()) == 0
+
+
 @pytest.mark.parametrize("flags", MQ)
 @pytest.mark.parametrize("spread", ["moderate", "extreme"])
 def test_verify_fp8_under_unequal_scales(oracle, flags, spread):
