@@ -538,7 +538,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         const float4 c4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16);
         const float4 a4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16 + 4);
         const float4 i4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16 + 8);
-        cq[0] = c4.x * rowc; cq[1] = c4.y * rowc; cq[2] = c4.z * rowc; cq[3] = c4.w * rowc;
+        // (kept above zero: a masked score, -inf, times 0 would be NaN)
+        cq[0] = fmaxf(c4.x * rowc, 1e-37f); cq[1] = fmaxf(c4.y * rowc, 1e-37f);
+        cq[2] = fmaxf(c4.z * rowc, 1e-37f); cq[3] = fmaxf(c4.w * rowc, 1e-37f);
         aq[0] = a4.x; aq[1] = a4.y; aq[2] = a4.z; aq[3] = a4.w;
         iq[0] = i4.x; iq[1] = i4.y; iq[2] = i4.z; iq[3] = i4.w;
         sc_stage += 2;
