@@ -66,6 +66,8 @@ extern "C" {
 
 #define PDA_FLAG_MQ_MMA_SYNC 2u   /* multi-query calls (verify, shared prefix): use the mma.sync
                                      kernel even where the tcgen05 + TMEM kernel applies */
+#define PDA_FLAG_MQ_PERSISTENT 4u /* paged_verify_attention, unsplit, bf16 head_dim 128: the tcgen05 kernel
+                                     with one persistent CTA per SM */
 
 typedef void* pda_stream_t; /* cudaStream_t */
 

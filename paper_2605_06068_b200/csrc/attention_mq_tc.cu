@@ -585,8 +585,10 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         // O and l may only be touched once the last PV into them has completed: PV(it-1), or (e4m3)
         // this set's PV(it-2). PV(it) is not issued before this warp arrives on bar_p below, and (bf16)
         // the other set rescales only after PV(it)
-        ok = kFp8 ? mbar_spin_bounded(my_pv, (k - 1) & 1)
-                  : mbar_spin_bounded(bar_pv + 8 * (set ^ 1), ((it - 1) >> 1) & 1);
+        // (a parity wait tells neighbouring phases apart only: first this set's own PV(it-2), after which
+        // the other set's barrier cannot be more than one phase behind)
+        ok = it >= 2 ? mbar_spin_bounded(my_pv, (k - 1) & 1) : true;
+        if (!kFp8 && ok) ok = mbar_spin_bounded(bar_pv + 8 * (set ^ 1), ((it - 1) >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
         tc_fence_after();
@@ -684,7 +686,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         if (ok) m_ref = m_sh[(last & 1) * kTcRows + t];
       }
       if (ok) {
-        ok = mbar_wait_bounded(bar_pv + 8 * (last & 1), (last >> 1) & 1);
+        // (the set that does not own the last iteration waits for its own last PV first: see above)
+        if ((last & 1) != set && last >= 1) ok = mbar_wait_bounded(my_pv, ((last - 1) >> 1) & 1);
+        if (ok) ok = mbar_wait_bounded(bar_pv + 8 * (last & 1), (last >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
       }
       if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);

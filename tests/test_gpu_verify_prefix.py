@@ -12,7 +12,8 @@ from util import DeviceWorkload, assert_close, bf16_tensor, bf16_to_bits, bf16_t
 pytestmark = pytest.mark.gpu
 
 # the multi-query kernels: tcgen05 + TMEM where it applies (bf16, head_dim 128), else / forced mma.sync
-MQ = [pytest.param(0, id="tcgen05"), pytest.param(pda.PDA_FLAG_MQ_MMA_SYNC, id="mma_sync")]
+MQ = [pytest.param(0, id="tcgen05"), pytest.param(pda.PDA_FLAG_MQ_MMA_SYNC, id="mma_sync"),
+      pytest.param(pda.PDA_FLAG_MQ_PERSISTENT, id="tcgen05_persistent")]
 
 
 def verify_inputs(w, T, seed):
@@ -107,7 +108,7 @@ def test_verify_batch_beyond_the_ranked_range(oracle, kv_dtype):
     else:
         ref, _ = oracle.paged_verify_attention(q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.scale,
                                                w.k_scale, w.v_scale)
-    for chunk in (0, 64):
+    for chunk, flags in ((0, 0), (64, 0), (0, pda.PDA_FLAG_MQ_PERSISTENT)):
         po = pl = None
         if chunk:
             mc = pda.max_chunks(int(lens.max()), chunk)
@@ -115,8 +116,8 @@ def test_verify_batch_beyond_the_ranked_range(oracle, kv_dtype):
             pl = torch.full((B, T, 32, mc), float("nan"), dtype=torch.float32, device="cuda")
         out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
                                          float(w.scale), chunk_tokens=chunk, part_o=po, part_lse=pl,
-                                         k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
-        assert_close(bf16_to_f64(out), ref, kv_dtype, what=f"verify batch {B} {kv_dtype} chunk {chunk}")
+                                         k_scale=dw.k_scale, v_scale=dw.v_scale, flags=flags, status=dw.status)
+        assert_close(bf16_to_f64(out), ref, kv_dtype, what=f"verify batch {B} {kv_dtype} chunk {chunk} flags {flags}")
     assert int(dw.status.item()) == 0
 
 
