@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libpda.so")
 PDA_BF16, PDA_FP8_E4M3 = 0, 1
 PDA_FLAG_FORCE_GENERIC = 1
 PDA_FLAG_MQ_MMA_SYNC = 2
-PDA_FLAG_MQ_PERSISTENT = 4
+PDA_FLAG_MQ_ONE_UNIT = 4
 DEV_STATUS = {0: "ok", 1: "bad page id", 2: "seq_len exceeds block table", 3: "copy wait timed out"}
 
 EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",

@@ -312,7 +312,7 @@ int paged_verify_attention(const void* q, const void* k_cache, const void* v_cac
   p.out = static_cast<__nv_bfloat16*>(out);
   pda::MqParams mp{p, n_query_tokens, 1, 0, max_chunks};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (!(flags & PDA_FLAG_MQ_MMA_SYNC) && (flags & PDA_FLAG_MQ_PERSISTENT) && pda::attention_mq_tcp_supports(mp)) {
+  if (!(flags & (PDA_FLAG_MQ_MMA_SYNC | PDA_FLAG_MQ_ONE_UNIT)) && pda::attention_mq_tcp_supports(mp)) {
     if (cudaError_t e = pda::launch_attention_mq_tcp(mp, s)) return static_cast<int>(e);
   } else if (!(flags & PDA_FLAG_MQ_MMA_SYNC) && pda::attention_mq_tc_supports(mp)) {
     if (cudaError_t e = pda::launch_attention_mq_tc(mp, s)) return static_cast<int>(e);

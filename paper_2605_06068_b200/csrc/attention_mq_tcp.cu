@@ -92,8 +92,8 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
       for (int w = 0; w < 4; ++w) mbar_init(bar_m + 8 * (4 * k + w), 1);  // per warp: rows w*32.. of set k
     }
-    mbar_init(bar_qready, kPSoftmaxWarps);  // a unit's Q is in tensor memory
-    mbar_init(bar_ofree, kPSoftmaxWarps);   // a unit's O and l have been read: the next unit's first PV may overwrite them
+    mbar_init(bar_qready, 4);               // a unit's Q is in tensor memory (stored by one softmax set)
+    mbar_init(bar_ofree, 4);                // a unit's O and l have been read (by the set that owns its last iteration)
     *cta_err = 0;
     fence_mbar_init();
     fence_proxy_async();
@@ -150,6 +150,18 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
       if (pos < 0) continue;
       const Unit u = unit_at(pos);
       const int32_t* table = p.block_table + static_cast<int64_t>(u.b) * p.block_table_stride;
+      // The producer reaches a unit some iterations before the softmax warps fetch its Q rows: it sends them
+      // towards L2 now (a load from DRAM takes about 3000 clocks while the other SMs stream).
+      if (u.n_iters > 0 && gi > 0) {
+        for (int rr = lane; rr < kPRows; rr += 32) {
+          const int r = u.rb * kPRows + rr;
+          if (r < rows_total) {
+            const __nv_bfloat16* row = p.q + ((static_cast<int64_t>(u.b) * T + r / G) * p.num_q_heads + u.g * G + (r % G)) * D;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(row + D / 2));
+          }
+        }
+      }
       int pg = 0;
       for (int it = 0; it < u.n_iters; ++it, ++gi) {
         const uint32_t s = gi % kPStages;
@@ -303,29 +315,44 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
       return -1;
     };
     // Q of a unit: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of
-    // S = Q . K^T; the two softmax warps that own the same 32 rows (w and w + 4) take half a row each
-    uint32_t qreg[32];  // 64 bf16 = 32 columns
-    auto fetch_q = [&](int k) {
+    // S = Q . K^T. One softmax set loads and stores the whole rows: at the end of a unit the set that does
+    // not own the last iteration, which is done one iteration earlier than the other (a load takes about
+    // 2500 clocks while the other SMs stream, from L2 as well as from DRAM).
+    auto load_q = [&](int k, uint32_t last_s) {
       const Unit u = unit_at(unit_pos(k, cta, n_ctas, n_units));
       const int r = u.rb * kPRows + t;
       const bool valid = r < rows_total;
       const int64_t qrow = (static_cast<int64_t>(u.b) * T + r / G) * p.num_q_heads + u.g * G + (r % G);
-      const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D) + set * 8;
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
+      uint32_t qreg[D / 2];
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
+      for (int ch = 0; ch < D / 8; ++ch) {
         const uint4 v = valid ? src[ch] : make_uint4(0u, 0u, 0u, 0u);
         qreg[4 * ch] = v.x; qreg[4 * ch + 1] = v.y; qreg[4 * ch + 2] = v.z; qreg[4 * ch + 3] = v.w;
       }
-    };
-    auto store_q = [&]() {
-      tmem_st32(tmem_q + lane_base + 32 * set, qreg);
-      tmem_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_tc(bar_qready);
+      bool ok = true;
+      if (last_s != 0xffffffffu) {  // the previous unit's last S has completed: its Q is no longer read
+        ok = mbar_spin_bounded(bar_s + 8 * (last_s & 1), (last_s >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+      }
+      if (ok) {
+#pragma unroll
+        for (int h = 0; h < D / 64; ++h) {
+          uint32_t part[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) part[j] = qreg[32 * h + j];
+          tmem_st32(tmem_q + lane_base + 32 * h, part);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_tc(bar_qready);
+      }
+      return ok;
     };
     int kn = next_unit(0);
-    if (kn >= 0) { fetch_q(kn); store_q(); }
+    if (kn >= 0 && set == 0) load_q(kn, 0xffffffffu);
     uint32_t gi0 = 0, uk = 0;  // first iteration of the unit; units with iterations so far
     for (int k = 0; k < n_rounds && alive; ++k) {
       const int pos = unit_pos(k, cta, n_ctas, n_units);
@@ -442,62 +469,46 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       if (!alive) break;
 
-      // ---- the unit's end. First the next unit's Q, so that its S is computed while this one drains:
-      // fetched now (this set has no more iterations here), stored once this unit's last S has completed.
+      // ---- the unit's end, shared out between the sets. The set that does not own the last iteration is
+      // done one iteration earlier: it loads the next unit's Q and goes on to that unit, whose first
+      // iteration is its own. The set that owns the last iteration waits for the last PV and writes the
+      // whole rows of the output while the other set is already at work on the next unit.
       const uint32_t glast = gi0 + u.n_iters - 1;
       bool ok = true;
-      if (kn >= 0) {
-        fetch_q(kn);
-        ok = mbar_spin_bounded(bar_s + 8 * (glast & 1), (glast >> 1) & 1);
+      if ((glast & 1) != static_cast<uint32_t>(set)) {
+        if (kn >= 0 && !load_q(kn, glast)) { fail(); break; }
+        // (the owner's last running maximum is not needed, but its barrier phase is consumed here: a parity
+        // wait only tells neighbouring phases apart)
+        ok = mbar_spin_bounded(bar_m + 8 * (4 * (glast & 1) + (warp & 3)), (glast >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { fail(); break; }
+      } else {
+        ok = mbar_spin_bounded(my_pv, (glast >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
         tc_fence_after();
-        store_q();
-      }
-      // the last iteration's reference (from the set that owned it) and the last PV
-      if ((glast & 1) != static_cast<uint32_t>(set)) {
-        ok = mbar_spin_bounded(bar_m + 8 * (4 * (glast & 1) + (warp & 3)), (glast >> 1) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (ok) m_ref = m_sh[(glast & 1) * kPRows + t];
-      }
-      if (ok) {
-        // (the set that does not own the last iteration waits for its own last PV first: a parity wait on the
-        // other set's barrier is only safe once that barrier is at most one phase behind)
-        if ((glast & 1) != static_cast<uint32_t>(set) && u.n_iters >= 2)
-          ok = mbar_spin_bounded(my_pv, ((glast - 1) >> 1) & 1);
-        if (ok) ok = mbar_spin_bounded(bar_pv + 8 * (glast & 1), (glast >> 1) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-      }
-      if (!ok) { fail(); break; }
-      tc_fence_after();
-      // l and this set's half of O into registers, then the accumulators are free for the next unit
-      uint32_t lv[32], o0[32], o1[32];
-      tmem_ld32(tmem_base + kPTmemL + lane_base, lv);
-      tmem_ld32(tmem_o + lane_base + 64 * set, o0);
-      tmem_ld32(tmem_o + lane_base + 64 * set + 32, o1);
-      tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_tc(bar_ofree);
-      const float l = __uint_as_float(lv[0]);
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      if (valid_row) {
-        uint4* dst = reinterpret_cast<uint4*>(p.out + qrow * D + (D / 2) * set);
+        uint32_t l_bits;
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(l_bits) : "r"(tmem_base + kPTmemL + lane_base));
+        tmem_wait_ld();
+        const float l = __uint_as_float(l_bits);
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        uint32_t w[D / 2];  // the row as bf16 pairs
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint32_t w[4];
+        for (int cb = 0; cb < D / 32; ++cb) {
+          uint32_t ov[32];
+          tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
+          tmem_wait_ld();
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            w[e] = pack2<false>(__uint_as_float(o0[8 * j + 2 * e]) * inv, __uint_as_float(o0[8 * j + 2 * e + 1]) * inv);
-          dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int j = 0; j < 16; ++j)
+            w[16 * cb + j] = pack2<false>(__uint_as_float(ov[2 * j]) * inv, __uint_as_float(ov[2 * j + 1]) * inv);
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_tc(bar_ofree);  // O and l are in registers: the next unit's first PV may overwrite them
+        if (valid_row) {
+          uint4* dst = reinterpret_cast<uint4*>(p.out + qrow * D);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            w[e] = pack2<false>(__uint_as_float(o1[8 * j + 2 * e]) * inv, __uint_as_float(o1[8 * j + 2 * e + 1]) * inv);
-          dst[4 + j] = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int j = 0; j < D / 8; ++j) dst[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         }
       }
       gi0 += u.n_iters;

@@ -88,7 +88,7 @@ def test_random_verification_blocks(oracle, seed):
         assert (bf16_to_bits(dw.k_cache) == k).all() and (bf16_to_bits(dw.v_cache) == v).all()
         ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
     what = f"seed {seed} Hq{Hq} kv{Hkv} D{D} {'e4m3' if fp8 else 'bf16'} T{T} lens {list(lens)}"
-    for flags in (0, pda.PDA_FLAG_MQ_MMA_SYNC, pda.PDA_FLAG_MQ_PERSISTENT):
+    for flags in (0, pda.PDA_FLAG_MQ_MMA_SYNC, pda.PDA_FLAG_MQ_ONE_UNIT):
         for chunk in (0, int(rng.choice([32, 64, 256]))):
             po = pl = None
             if chunk:

@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 # the multi-query kernels: tcgen05 + TMEM where it applies (bf16, head_dim 128), else / forced mma.sync
 MQ = [pytest.param(0, id="tcgen05"), pytest.param(pda.PDA_FLAG_MQ_MMA_SYNC, id="mma_sync"),
-      pytest.param(pda.PDA_FLAG_MQ_PERSISTENT, id="tcgen05_persistent")]
+      pytest.param(pda.PDA_FLAG_MQ_ONE_UNIT, id="tcgen05_one_unit")]
 
 
 def verify_inputs(w, T, seed):
@@ -108,7 +108,7 @@ def test_verify_batch_beyond_the_ranked_range(oracle, kv_dtype):
     else:
         ref, _ = oracle.paged_verify_attention(q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.scale,
                                                w.k_scale, w.v_scale)
-    for chunk, flags in ((0, 0), (64, 0), (0, pda.PDA_FLAG_MQ_PERSISTENT)):
+    for chunk, flags in ((0, 0), (64, 0), (0, pda.PDA_FLAG_MQ_ONE_UNIT)):
         po = pl = None
         if chunk:
             mc = pda.max_chunks(int(lens.max()), chunk)
