@@ -90,6 +90,41 @@ def test_verify_attention_fp8_and_causal_needle(oracle):
     assert np.abs(out[0, :-1]).max() < 3.0    # N(0,1) averages, nowhere near 1..128
 
 
+@pytest.mark.parametrize("flags", MQ)
+def test_verify_bad_table_entries_and_lengths_set_status(oracle, flags):
+    """A page id outside the pool and a length beyond the block table: the status word reports them (the
+    larger code wins), nothing is read outside the caches, and the other sequences' rows are right."""
+    lens = [300, 90, 200, 47, 130, 64]
+    T = 4
+    w = W.make_workload("bad", lens, 32, 8, 128, seed=61)
+    q, kn, vn = verify_inputs(w, T, 62)
+    k, v = w.k_cache.copy(), w.v_cache.copy()
+    oracle.kv_append_tokens(kn, vn, k, v, w.block_table, w.seq_lens)
+    ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
+    dw = DeviceWorkload(w)
+    pda.kv_append_tokens(bf16_tensor(kn), bf16_tensor(vn), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens)
+    bt = dw.block_table.clone()
+    bt[1, 2] = w.num_pages + 7      # sequence 1: a page id past the pool
+    bt[4, 0] = -1                   # sequence 4: a negative page id
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, bt, dw.seq_lens, float(w.scale),
+                                     flags=flags, status=st)
+    got = bf16_to_f64(out)
+    assert int(st.item()) == 1      # PDA_DEV_BAD_PAGE
+    assert np.isfinite(got[[0, 2, 3, 5]]).all()
+    for b in (0, 2, 3, 5):
+        assert_close(got[b:b + 1], ref[b:b + 1], what=f"sequence {b} beside a bad table row, flags {flags}")
+    sl = dw.seq_lens.clone()
+    sl[2] = bt.shape[1] * 16 + 5    # sequence 2: longer than its table row can describe
+    st.zero_()
+    out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, sl, float(w.scale),
+                                     flags=flags, status=st)
+    got = bf16_to_f64(out)
+    assert int(st.item()) == 2      # PDA_DEV_BAD_SEQ_LEN
+    for b in (0, 1, 3, 4, 5):
+        assert_close(got[b:b + 1], ref[b:b + 1], what=f"sequence {b} beside a bad length, flags {flags}")
+
+
 @pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
 def test_verify_batch_beyond_the_ranked_range(oracle, kv_dtype):
     """More than 128 sequences: the CTAs take the sequences in index order instead of longest first;
