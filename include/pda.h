@@ -221,7 +221,11 @@ int kv_append_tokens_fp8(const void* k_new, const void* v_new, void* k_cache, vo
  * PDA_FLAG_MQ_MMA_SYNC selects the mma.sync kernel instead. Unsplit calls on bf16
  * caches with head_dim 128 and up to 1024 sequences run as one persistent CTA per SM
  * that walks through the (sequence, kv head, row block) units, longest sequences
- * first (PDA_FLAG_MQ_ONE_UNIT: one CTA per unit).
+ * first (PDA_FLAG_MQ_ONE_UNIT: one CTA per unit). That kernel shares out its last
+ * units through a counter in device memory which the library owns (a pool of 64,
+ * taken in turn by the launches and left at zero by each): up to 64 such launches
+ * may be in flight at once on a device; a launch captured in a CUDA graph keeps its
+ * counter, so one graph must not run beside itself on two streams.
  * e4m3 on tcgen05: the products are e4m3 x e4m3 on the cache's bytes; q and the softmax
  * weights enter as two 8-bit parts each (q to 2^-8, a weight to 2^-7 relative), the
  * page scales through the softmax. An output element is within about 0.3 % of the

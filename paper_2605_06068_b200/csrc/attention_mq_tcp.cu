@@ -8,10 +8,14 @@
 //   - the next unit's Q rows are fetched during the current unit's last iterations and stored to tensor
 //     memory as soon as its last S has completed, so the S of the next unit is computed while the last
 //     P.V and the output of the current one are under way.
-// Units are dealt to the CTAs in serpentine order over the sequences sorted by length (longest first),
-// all of a sequence's units next to one another: every CTA gets a like share without a global counter.
+// Units are claimed from a counter in device memory in the order of the sequences sorted by length (longest
+// first; all of a sequence's units next to one another), so a CTA that drew long units draws fewer. The
+// counter is one of a small pool the library owns; the CTA that leaves last puts it back to zero.
 // Iterations are numbered through all units of a CTA (gi); ring stages, S/P buffers, softmax sets and
 // barrier phases follow gi as they follow the iteration index in the one-unit kernel.
+#include <atomic>
+#include <mutex>
+
 #include "common.cuh"
 #include "tma_ptx.cuh"
 #include "tcgen05_ptx.cuh"
@@ -33,22 +37,43 @@ constexpr int kPMBytes = 2 * kPRows * 4;                     // running row maxi
 constexpr int kPMaxBatch = 1024;                             // lengths and order of the sequences in shared memory
 constexpr int kPSortBatch = 352;                             // sorted up to one sequence per thread
 constexpr int kPLensBytes = kPMaxBatch * 4, kPOrderBytes = kPMaxBatch * 2;
-constexpr int kPSmemBytes = kPStages * kPStageBytes + kPOnesBytes + kPMBytes + kPLensBytes + kPOrderBytes + 512 + 1024;
+constexpr int kPSmemBytes = kPStages * kPStageBytes + kPOnesBytes + kPMBytes + kPLensBytes + kPOrderBytes + 128 + 512 + 1024;
 constexpr int kPSoftmaxWarps = 8, kPProducerWarp = 8, kPMmaWarp = 9, kPPvWarp = 10;
 constexpr int kPThreads = 352;
 constexpr uint32_t kPTmemCols = 512;
 constexpr uint32_t kPTmemO = 128, kPTmemQ = 256, kPTmemP = 320, kPTmemL = 384;
 constexpr float kPRescaleThreshold = 8.f;
 
-// The k-th unit of CTA `cta`: position in the dealt order, or -1 past the end.
-__device__ __forceinline__ int unit_pos(int k, int cta, int n_ctas, int n_units) {
-  const int pos = k * n_ctas + ((k & 1) ? n_ctas - 1 - cta : cta);
-  return pos < n_units ? pos : -1;
+// Units are claimed from a counter in device memory (longest sequences first) by the producer warp, which
+// is the first to need them, and handed to the other warps through a small ring in shared memory: entry k
+// holds the position of the CTA's k-th unit in the sorted order, or -1 when there are no more. Only units
+// with iterations go through the ring (the producer writes the zero rows of an empty sequence itself), so
+// the producer is never more than kPStages + 2 entries ahead of the slowest reader.
+constexpr int kPClaimRing = 16;
+constexpr int kPClaimedRounds = 3;
+__device__ __forceinline__ void publish_unit(volatile int* ring_sh, int k, int pos) {  // one thread
+  ring_sh[2 * (k % kPClaimRing) + 1] = pos;
+  __threadfence_block();
+  ring_sh[2 * (k % kPClaimRing)] = k + 1;  // tag: entry k is valid
+}
+__device__ __forceinline__ int unit_entry(volatile int* ring_sh, int k, int lane) {  // a whole warp; -2: timed out
+  int pos = -2;
+  if (lane == 0) {
+    for (uint32_t i = 0; i < (1u << 24); ++i) {
+      if (ring_sh[2 * (k % kPClaimRing)] == k + 1) {
+        __threadfence_block();
+        pos = ring_sh[2 * (k % kPClaimRing) + 1];
+        break;
+      }
+      __nanosleep(64);
+    }
+  }
+  return __shfl_sync(0xffffffffu, pos, 0);
 }
 
 __global__ void __launch_bounds__(kPThreads, 1)
 attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
-                        const __grid_constant__ CUtensorMap v_map, MqParams mp) {
+                        const __grid_constant__ CUtensorMap v_map, MqParams mp, unsigned int* claim) {
   const AttnParams& p = mp.a;
   constexpr int D = kPD;
   extern __shared__ uint8_t smem_raw[];
@@ -57,8 +82,9 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
   float* m_sh = reinterpret_cast<float*>(ones_smem + kPOnesBytes);              // [2][128]
   int* lens_sh = reinterpret_cast<int*>(m_sh + 2 * kPRows);                      // [batch]
   uint16_t* order_sh = reinterpret_cast<uint16_t*>(lens_sh + kPMaxBatch);        // [batch]: longest first
+  int* ring_sh = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(order_sh) + kPOrderBytes);  // [kPClaimRing][tag, position]
   // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2][4], qready, ofree
-  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(order_sh) + kPOrderBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring_sh + 2 * kPClaimRing);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kPStages + 18);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
 
@@ -69,8 +95,19 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
   const int per_seq = p.geom.num_kv_heads * n_rb;   // units of a sequence
   const int n_units = p.batch * per_seq;
   const int cta = blockIdx.x, n_ctas = gridDim.x;
+  // The claim counter is zero between launches: the CTA that leaves last puts it back.
+  auto leave = [&]() {
+    if (threadIdx.x == 0 && atomicAdd(&claim[1], 1u) == gridDim.x - 1) {
+      claim[0] = 0u;
+      claim[1] = 0u;
+      __threadfence();
+    }
+  };
   // once any CTA of this launch has reported a timed-out wait, the rest do not start
-  if (p.status != nullptr && *reinterpret_cast<volatile int32_t*>(p.status) == PDA_DEV_TIMEOUT) return;
+  if (p.status != nullptr && *reinterpret_cast<volatile int32_t*>(p.status) == PDA_DEV_TIMEOUT) {
+    leave();
+    return;
+  }
 
   const uint32_t ring = smem_u32(smem);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kPStages;
@@ -94,6 +131,7 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
     }
     mbar_init(bar_qready, 4);               // a unit's Q is in tensor memory (stored by one softmax set)
     mbar_init(bar_ofree, 4);                // a unit's O and l have been read (by the set that owns its last iteration)
+    for (int i = 0; i < 2 * kPClaimRing; ++i) ring_sh[i] = 0;
     *cta_err = 0;
     fence_mbar_init();
     fence_proxy_async();
@@ -138,21 +176,52 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
     u.n_iters = (u.n_pages + kPPagesPerIter - 1) / kPPagesPerIter;
     return u;
   };
-  const int n_rounds = (n_units + n_ctas - 1) / n_ctas;
 
   if (warp == kPProducerWarp) {
     // ================= TMA producer: runs through the units' tiles, up to kPStages iterations ahead ====
     const uint32_t leader = elect_one();
     bool bad = false, dead = false;
     uint32_t gi = 0;
-    for (int k = 0; k < n_rounds && !dead; ++k) {
-      const int pos = unit_pos(k, cta, n_ctas, n_units);
-      if (pos < 0) continue;
+    // (a quarter of the rounds, at most kPClaimedRounds: with only three or four units a CTA the deal is as
+    // even as claiming, and claiming would make every CTA work on units of like length at any one time)
+    const int dealt_rounds = n_units / n_ctas - min(kPClaimedRounds, n_units / n_ctas / 4);
+    int n_dealt = 0;
+    for (int k = 0; !dead;) {
+      // The first rounds are dealt in serpentine order over the sorted units (every CTA works on a mix of long
+      // and short units, which keeps the HBM busy while some CTAs are between units); the shortest units, the
+      // last kPClaimedRounds rounds' worth, are claimed from the counter and even out the CTAs' ends.
+      int pos = 0;
+      if (n_dealt < dealt_rounds) {
+        pos = n_dealt * n_ctas + ((n_dealt & 1) ? n_ctas - 1 - cta : cta);
+        ++n_dealt;
+      } else {
+        if (lane == 0) pos = dealt_rounds * n_ctas + static_cast<int>(atomicAdd(&claim[0], 1u));
+        pos = __shfl_sync(0xffffffffu, pos, 0);
+      }
+      if (pos >= n_units) {
+        if (lane == 0) publish_unit(ring_sh, k, -1);
+        break;
+      }
       const Unit u = unit_at(pos);
+      if (u.n_iters == 0) {  // an empty (or misdescribed) sequence: its output rows are zero, written here
+        if (u.bad && lane == 0) report(p.status, PDA_DEV_BAD_SEQ_LEN);
+        for (int rr = lane; rr < kPRows; rr += 32) {
+          const int r = u.rb * kPRows + rr;
+          if (r < rows_total) {
+            uint4* dst = reinterpret_cast<uint4*>(
+                p.out + ((static_cast<int64_t>(u.b) * T + r / G) * p.num_q_heads + u.g * G + (r % G)) * D);
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j) dst[j] = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+        continue;
+      }
+      if (lane == 0) publish_unit(ring_sh, k, pos);
+      ++k;
       const int32_t* table = p.block_table + static_cast<int64_t>(u.b) * p.block_table_stride;
       // The producer reaches a unit some iterations before the softmax warps fetch its Q rows: it sends them
       // towards L2 now (a load from DRAM takes about 3000 clocks while the other SMs stream).
-      if (u.n_iters > 0 && gi > 0) {
+      if (gi > 0) {
         for (int rr = lane; rr < kPRows; rr += 32) {
           const int r = u.rb * kPRows + rr;
           if (r < rows_total) {
@@ -204,14 +273,13 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
     const uint32_t leader = elect_one();
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
     bool ok = true;
-    uint32_t gi = 0, uk = 0;
-    for (int k = 0; k < n_rounds && ok; ++k) {
-      const int pos = unit_pos(k, cta, n_ctas, n_units);
-      if (pos < 0) continue;
+    uint32_t gi = 0;
+    for (int k = 0; ok; ++k) {
+      const int pos = unit_entry(ring_sh, k, lane);
+      if (pos < 0) { ok = pos == -1; break; }
       const Unit u = unit_at(pos);
-      if (u.n_iters == 0) continue;
       // this unit's Q is in tensor memory (the softmax warps store it once the previous unit's last S is done)
-      ok = mbar_wait_bounded(bar_qready, uk & 1);
+      ok = mbar_wait_bounded(bar_qready, k & 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -247,7 +315,6 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
         }
         tc_commit_if(leader, bar_s + 8 * (gi & 1));
       }
-      ++uk;
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   } else if (warp == kPPvWarp) {
@@ -258,15 +325,15 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
     const uint32_t leader = elect_one();
     const uint32_t u_tmem = __shfl_sync(0xffffffffu, tmem_base, 0);
     bool ok = true;
-    uint32_t gi = 0, uk = 0;  // units with iterations so far
-    for (int k = 0; k < n_rounds && ok; ++k) {
-      const int pos = unit_pos(k, cta, n_ctas, n_units);
-      if (pos < 0) continue;
+    uint32_t gi = 0;
+    for (int k = 0; ok; ++k) {
+      const int pos = unit_entry(ring_sh, k, lane);
+      if (pos < 0) { ok = pos == -1; break; }
       const Unit u = unit_at(pos);
       for (int it = 0; it < u.n_iters; ++it, ++gi) {
         ok = mbar_wait_bounded(bar_p + 8 * (gi & 1), (gi >> 1) & 1);
         // the unit's first PV overwrites O and l: every softmax warp has read the previous unit's
-        if (ok && it == 0 && uk > 0) ok = mbar_wait_bounded(bar_ofree, (uk - 1) & 1);
+        if (ok && it == 0 && k > 0) ok = mbar_wait_bounded(bar_ofree, (k - 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -292,7 +359,6 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
         tc_commit_if(leader, empty0 + 8 * stage_i);     // the stage may be refilled once these MMAs have read it
         tc_commit_if(leader, bar_pv + 8 * (gi & 1));    // O and l updated, P buffer free again
       }
-      if (u.n_iters > 0) ++uk;
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   } else {
@@ -306,20 +372,12 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
     const uint32_t my_m = bar_m + 8 * (4 * set + (warp & 3)), other_m = bar_m + 8 * (4 * (set ^ 1) + (warp & 3));
     bool alive = true;
     auto fail = [&]() { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; };
-    // the first unit at or after round k that has iterations, or -1
-    auto next_unit = [&](int k) {
-      for (; k < n_rounds; ++k) {
-        const int pos = unit_pos(k, cta, n_ctas, n_units);
-        if (pos >= 0 && unit_at(pos).n_iters > 0) return k;
-      }
-      return -1;
-    };
     // Q of a unit: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of
     // S = Q . K^T. One softmax set loads and stores the whole rows: at the end of a unit the set that does
     // not own the last iteration, which is done one iteration earlier than the other (a load takes about
     // 2500 clocks while the other SMs stream, from L2 as well as from DRAM).
-    auto load_q = [&](int k, uint32_t last_s) {
-      const Unit u = unit_at(unit_pos(k, cta, n_ctas, n_units));
+    auto load_q = [&](int pos_q, uint32_t last_s) {
+      const Unit u = unit_at(pos_q);
       const int r = u.rb * kPRows + t;
       const bool valid = r < rows_total;
       const int64_t qrow = (static_cast<int64_t>(u.b) * T + r / G) * p.num_q_heads + u.g * G + (r % G);
@@ -351,29 +409,18 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       return ok;
     };
-    int kn = next_unit(0);
-    if (kn >= 0 && set == 0) load_q(kn, 0xffffffffu);
-    uint32_t gi0 = 0, uk = 0;  // first iteration of the unit; units with iterations so far
-    for (int k = 0; k < n_rounds && alive; ++k) {
-      const int pos = unit_pos(k, cta, n_ctas, n_units);
-      if (pos < 0) continue;
+    int pos = unit_entry(ring_sh, 0, lane);  // the CTA's first unit
+    if (pos == -2) fail();
+    if (pos >= 0 && set == 0) load_q(pos, 0xffffffffu);
+    uint32_t gi0 = 0;  // first iteration of the unit
+    for (int k = 0; alive && pos >= 0; ++k) {
       const Unit u = unit_at(pos);
       const int r = u.rb * kPRows + t;
       const bool valid_row = r < rows_total;
       const int i_tok = r / G;
       const int64_t qrow = (static_cast<int64_t>(u.b) * T + i_tok) * p.num_q_heads + u.g * G + (r % G);
-      if (u.n_iters == 0) {  // an empty (or misdescribed) sequence: its output rows are zero
-        if (u.bad && tid == 0) report(p.status, PDA_DEV_BAD_SEQ_LEN);
-        if (valid_row) {
-          uint4* dst = reinterpret_cast<uint4*>(p.out + qrow * D + (D / 2) * set);
-#pragma unroll
-          for (int j = 0; j < D / 16; ++j) dst[j] = make_uint4(0u, 0u, 0u, 0u);
-        }
-        continue;
-      }
       const int L = u.L;
       const int lim = mp.causal ? min(L, L - T + i_tok + 1) : L;
-      kn = next_unit(k + 1);
       float m_ref = -INFINITY;   // reference max the accumulated O and l (both in tensor memory) are scaled by
       for (int it = ((gi0 & 1u) == static_cast<uint32_t>(set)) ? 0 : 1; it < u.n_iters; it += 2) {
         const uint32_t gi = gi0 + it;
@@ -475,8 +522,10 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
       // whole rows of the output while the other set is already at work on the next unit.
       const uint32_t glast = gi0 + u.n_iters - 1;
       bool ok = true;
+      int pos_next;  // the CTA's next unit (claimed by the producer some iterations ago), or -1
       if ((glast & 1) != static_cast<uint32_t>(set)) {
-        if (kn >= 0 && !load_q(kn, glast)) { fail(); break; }
+        pos_next = unit_entry(ring_sh, k + 1, lane);
+        if (pos_next == -2 || (pos_next >= 0 && !load_q(pos_next, glast))) { fail(); break; }
         // (the owner's last running maximum is not needed, but its barrier phase is consumed here: a parity
         // wait only tells neighbouring phases apart)
         ok = mbar_spin_bounded(bar_m + 8 * (4 * (glast & 1) + (warp & 3)), (glast >> 1) & 1);
@@ -510,11 +559,12 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
           for (int j = 0; j < D / 8; ++j) dst[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         }
+        pos_next = unit_entry(ring_sh, k + 1, lane);
+        if (pos_next == -2) { fail(); break; }
       }
       gi0 += u.n_iters;
-      ++uk;
+      pos = pos_next;
     }
-    (void)uk;
   }
 
   // ---- teardown: everyone is done with tensor memory before it is released
@@ -525,6 +575,7 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kPTmemCols) : "memory");
   }
+  leave();
 }
 
 }  // namespace
@@ -537,6 +588,30 @@ bool attention_mq_tcp_supports(const MqParams& mp) {
   if (!(p.scale > 0.f) || !(p.scale < INFINITY)) return false;  // the row maximum is taken before scaling
   return true;
 }
+
+namespace {
+// Claim counters: [next unit, CTAs that have left] each, zero between launches. Launches take the slots in
+// turn, so that launches running side by side on different streams do not share one (up to kClaimSlots of
+// them); a captured launch keeps the slot it was captured with.
+constexpr int kClaimSlots = 64, kClaimDevices = 64;
+__device__ unsigned int g_claim[kClaimSlots][4];
+std::atomic<unsigned> g_claim_next{0};
+std::mutex g_claim_mu;
+unsigned int* g_claim_base[kClaimDevices] = {};
+cudaError_t claim_counter(int dev, unsigned int** out) {
+  if (dev < 0 || dev >= kClaimDevices) return cudaErrorInvalidDevice;
+  {
+    std::lock_guard<std::mutex> lock(g_claim_mu);
+    if (g_claim_base[dev] == nullptr) {
+      void* ptr = nullptr;
+      if (cudaError_t e = cudaGetSymbolAddress(&ptr, g_claim)) return e;
+      g_claim_base[dev] = static_cast<unsigned int*>(ptr);
+    }
+  }
+  *out = g_claim_base[dev] + 4 * (g_claim_next.fetch_add(1) % kClaimSlots);
+  return cudaSuccess;
+}
+}  // namespace
 
 cudaError_t launch_attention_mq_tcp(const MqParams& mp, cudaStream_t stream) {
   const AttnParams& p = mp.a;
@@ -555,8 +630,12 @@ cudaError_t launch_attention_mq_tcp(const MqParams& mp, cudaStream_t stream) {
   const int rows_total = mp.n_q * p.group;
   const int n_rb = (rows_total + kPRows - 1) / kPRows;
   const int64_t n_units = static_cast<int64_t>(p.batch) * p.geom.num_kv_heads * n_rb;
+  // with a unit or less per SM there is nothing to carry from one unit to the next
+  if (n_units <= sms && attention_mq_tc_supports(mp)) return launch_attention_mq_tc(mp, stream);
   const unsigned grid = static_cast<unsigned>(n_units < sms ? n_units : sms);
-  attention_mq_tcp_kernel<<<grid, kPThreads, kPSmemBytes, stream>>>(k_map, v_map, mp);
+  unsigned int* claim = nullptr;
+  if ((e = claim_counter(dev, &claim)) != cudaSuccess) return e;
+  attention_mq_tcp_kernel<<<grid, kPThreads, kPSmemBytes, stream>>>(k_map, v_map, mp, claim);
   return cudaGetLastError();
 }
 

@@ -90,11 +90,34 @@ def test_verify_attention_fp8_and_causal_needle(oracle):
     assert np.abs(out[0, :-1]).max() < 3.0    # N(0,1) averages, nowhere near 1..128
 
 
+@pytest.mark.parametrize("T", [1, 16, 40])
+def test_verify_more_units_than_sms(oracle, T):
+    """Enough (sequence, kv head, row block) units that the persistent kernel carries several per CTA: units
+    of one iteration and of many, odd page counts, ragged tails, one and two row blocks, and (T = 16) a share
+    of the units claimed from the counter rather than dealt."""
+    rng = np.random.default_rng(300 + T)
+    B = 40 if T != 16 else 90
+    lens = np.maximum(rng.integers(1, 900, size=B), T)
+    lens[:4] = [T, 64, 65, 128]
+    w = W.make_workload("many_units", lens, 32, 8, 128, seed=301 + T)
+    q, kn, vn = verify_inputs(w, T, 302 + T)
+    k, v = w.k_cache.copy(), w.v_cache.copy()
+    oracle.kv_append_tokens(kn, vn, k, v, w.block_table, w.seq_lens)
+    ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
+    dw = DeviceWorkload(w)
+    pda.kv_append_tokens(bf16_tensor(kn), bf16_tensor(vn), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens)
+    for rep in range(3):   # repeated launches: the claim counter is back at zero each time
+        out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                         float(w.scale), status=dw.status)
+        assert_close(bf16_to_f64(out), ref, what=f"verify, {B * 8} units, T={T}, launch {rep}")
+    assert int(dw.status.item()) == 0
+
+
 @pytest.mark.parametrize("flags", MQ)
 def test_verify_bad_table_entries_and_lengths_set_status(oracle, flags):
     """A page id outside the pool and a length beyond the block table: the status word reports them (the
     larger code wins), nothing is read outside the caches, and the other sequences' rows are right."""
-    lens = [300, 90, 200, 47, 130, 64]
+    lens = [300, 90, 200, 47, 130, 64] + [40 + 7 * i for i in range(18)]   # 24 x 8 units: more than SMs
     T = 4
     w = W.make_workload("bad", lens, 32, 8, 128, seed=61)
     q, kn, vn = verify_inputs(w, T, 62)
@@ -111,8 +134,9 @@ def test_verify_bad_table_entries_and_lengths_set_status(oracle, flags):
                                      flags=flags, status=st)
     got = bf16_to_f64(out)
     assert int(st.item()) == 1      # PDA_DEV_BAD_PAGE
-    assert np.isfinite(got[[0, 2, 3, 5]]).all()
-    for b in (0, 2, 3, 5):
+    good = [b for b in range(len(lens)) if b not in (1, 4)]
+    assert np.isfinite(got[good]).all()
+    for b in good:
         assert_close(got[b:b + 1], ref[b:b + 1], what=f"sequence {b} beside a bad table row, flags {flags}")
     sl = dw.seq_lens.clone()
     sl[2] = bt.shape[1] * 16 + 5    # sequence 2: longer than its table row can describe
@@ -121,8 +145,9 @@ def test_verify_bad_table_entries_and_lengths_set_status(oracle, flags):
                                      flags=flags, status=st)
     got = bf16_to_f64(out)
     assert int(st.item()) == 2      # PDA_DEV_BAD_SEQ_LEN
-    for b in (0, 1, 3, 4, 5):
+    for b in [b for b in range(len(lens)) if b != 2]:
         assert_close(got[b:b + 1], ref[b:b + 1], what=f"sequence {b} beside a bad length, flags {flags}")
+    assert (got[2] == 0).all()      # the misdescribed sequence's rows are zero
 
 
 @pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
