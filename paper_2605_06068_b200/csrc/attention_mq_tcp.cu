@@ -8,9 +8,11 @@
 //   - the next unit's Q rows are fetched during the current unit's last iterations and stored to tensor
 //     memory as soon as its last S has completed, so the S of the next unit is computed while the last
 //     P.V and the output of the current one are under way.
-// Units are claimed from a counter in device memory in the order of the sequences sorted by length (longest
-// first; all of a sequence's units next to one another), so a CTA that drew long units draws fewer. The
-// counter is one of a small pool the library owns; the CTA that leaves last puts it back to zero.
+// Units are ordered by the length of their sequence (longest first; all of a sequence's units next to one
+// another). Most are dealt to the CTAs in serpentine order, so that every CTA works on a mix of long and
+// short units; the shortest ones are claimed from a counter in device memory, so that a CTA whose share
+// was long draws fewer of them. The counter is one of a small pool the library owns; the CTA that leaves
+// last puts it back to zero.
 // Iterations are numbered through all units of a CTA (gi); ring stages, S/P buffers, softmax sets and
 // barrier phases follow gi as they follow the iteration index in the one-unit kernel.
 #include <atomic>
