@@ -298,3 +298,43 @@ def test_shared_prefix_cascade_in_a_cuda_graph(oracle):
         torch.cuda.synchronize()
         assert torch.equal(out.view(torch.int16), eager.view(torch.int16))
     assert int(dw.status.item()) == 0
+
+
+def test_verify_persistent_kernel_in_a_cuda_graph(oracle):
+    """The persistent kernel shares out its last units through a counter the library owns; a captured launch
+    keeps its counter, which every replay must find at zero and leave at zero."""
+    rng = np.random.default_rng(401)
+    B, T = 120, 8
+    lens = np.maximum(rng.integers(1, 700, size=B), T)
+    w = W.make_workload("graph_units", lens, 32, 8, 128, seed=402)
+    q, kn, vn = verify_inputs(w, T, 403)
+    k, v = w.k_cache.copy(), w.v_cache.copy()
+    oracle.kv_append_tokens(kn, vn, k, v, w.block_table, w.seq_lens)
+    ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
+    dw = DeviceWorkload(w)
+    pda.kv_append_tokens(bf16_tensor(kn), bf16_tensor(vn), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens)
+    dq = bf16_tensor(q)
+    out = torch.empty_like(dq)
+
+    def run(stream=None):
+        pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, float(w.scale),
+                                   out=out, status=dw.status, stream=stream)
+    run()
+    torch.cuda.synchronize()
+    eager = out.clone()
+    assert_close(bf16_to_f64(eager), ref, what="verify eager")
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            run(s)
+    for _ in range(3):
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), eager.view(torch.int16))
+        run()                  # eager launches between the replays take other counters
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), eager.view(torch.int16))
+    assert int(dw.status.item()) == 0
