@@ -199,6 +199,8 @@ def run_gpu(args):
 
     w = make(args.workload, rank)
     chunk = DEFAULT_CHUNK[w.name] if args.chunk is None else args.chunk
+    if args.chunk is None and args.mode == "verify" and chunk:
+        chunk *= 2   # a multi-query unit costs more to start than a decode unit: larger chunks (4096 for longctx)
     dev = torch.device("cuda", local)
     to16 = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
     q = to16(w.q)
