@@ -55,3 +55,34 @@ def test_full_size_config(oracle, name, chunk, chunk_sep):
     worst, nerr = assert_close(got, ref, w.kv_dtype, what=f"{name} separate chunk {chunk_sep}")
     print(f"{name}: separate chunk {chunk_sep}: max err/tol {worst:.3f}, max err/rms {nerr:.3e}")
     assert int(dw.status.item()) == 0
+
+
+@pytest.mark.parametrize("name", ["llama8b", "chat70b", "prefix_fp8"])
+def test_full_size_verification_sampled(oracle, name):
+    """16-token verification at the full size of a workload, in the configuration `bench.py --mode verify`
+    times (unsplit; the persistent tcgen05 kernel for bf16, with chat70b's 2048 units partly claimed from the
+    counter; the e4m3 tensor-core kernel for prefix_fp8), against the oracle on a sample of the sequences:
+    the longest, the shortest and ten others."""
+    T = 16
+    w = W.WORKLOADS[name]()
+    rng = np.random.default_rng(77)
+    q = W.f32_to_bf16_bits(rng.standard_normal((w.batch, T, w.num_q_heads, w.head_dim), dtype=np.float32))
+    dw = DeviceWorkload(w)
+    k, v = w.k_cache, w.v_cache
+    if w.kv_dtype == "bf16":   # (a bf16 workload's last slots are filled by the append)
+        k, v = host_appended(oracle, w)
+        dw.append()
+    out = pda.paged_verify_attention(torch.from_numpy(q.view(np.int16)).cuda().view(torch.bfloat16), dw.k_cache,
+                                     dw.v_cache, dw.block_table, dw.seq_lens, float(w.scale),
+                                     k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+    got = bf16_to_f64(out)
+    assert int(dw.status.item()) == 0
+    order = np.argsort(w.seq_lens)
+    pick = np.unique(np.concatenate([order[:1], order[-1:], rng.choice(w.batch, size=10, replace=False)]))
+    scales = (w.k_scale, w.v_scale) if w.kv_dtype == "e4m3" else ()
+    ref, _ = oracle.paged_verify_attention(q[pick], k, v, w.block_table[pick], w.seq_lens[pick], w.scale, *scales)
+    worst, nerr = assert_close(got[pick], ref, w.kv_dtype, what=f"{name} verification of {T} tokens, sampled")
+    print(f"{name}: verify {T}: max err/tol {worst:.3f}, max err/rms {nerr:.3e}")
+    # every other sequence: finite and of the same scale as the sampled ones
+    assert np.isfinite(got).all()
+    assert np.sqrt((got ** 2).mean()) > 0.3 * np.sqrt((ref ** 2).mean())
