@@ -86,3 +86,30 @@ def test_full_size_verification_sampled(oracle, name):
     # every other sequence: finite and of the same scale as the sampled ones
     assert np.isfinite(got).all()
     assert np.sqrt((got ** 2).mean()) > 0.3 * np.sqrt((ref ** 2).mean())
+
+
+@pytest.mark.parametrize("name,prefix,pchunk,chunk", [("scenario_c", 32768, 2048, 256), ("prefix_fp8", 2048, 512, 256)])
+def test_full_size_shared_prefix_cascade_sampled(oracle, name, prefix, pchunk, chunk):
+    """The shared-prefix cascade at full size, with the chunk sizes `bench.py --mode cascade` uses, against
+    the plain oracle (the cascade is an exact reorganisation of decode attention) on sampled sequences."""
+    w = W.WORKLOADS[name]()
+    dw = DeviceWorkload(w)
+    k, v = w.k_cache, w.v_cache
+    if w.kv_dtype == "bf16":
+        k, v = host_appended(oracle, w)
+        dw.append()
+    mc = (prefix + pchunk - 1) // pchunk + pda.max_chunks(int(w.seq_lens.max()) - prefix + 1, chunk)
+    po = torch.full((w.batch, w.num_q_heads, mc, w.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    pl = torch.full((w.batch, w.num_q_heads, mc), float("nan"), dtype=torch.float32, device="cuda")
+    out = pda.paged_prefix_decode_attention(dw.q, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                            float(w.scale), prefix, pchunk, chunk, po, pl,
+                                            k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+    got = bf16_to_f64(out)
+    assert int(dw.status.item()) == 0 and np.isfinite(got).all()
+    rng = np.random.default_rng(78)
+    order = np.argsort(w.seq_lens)
+    pick = np.unique(np.concatenate([order[:1], order[-1:], rng.choice(w.batch, size=4, replace=False)]))
+    scales = (w.k_scale, w.v_scale) if w.kv_dtype == "e4m3" else ()
+    ref, _ = oracle.paged_decode_attention(w.q[pick], k, v, w.block_table[pick], w.seq_lens[pick], w.scale, *scales)
+    worst, nerr = assert_close(got[pick], ref, w.kv_dtype, what=f"{name} cascade, sampled")
+    print(f"{name}: cascade {pchunk}/{chunk}: max err/tol {worst:.3f}, max err/rms {nerr:.3e}")
