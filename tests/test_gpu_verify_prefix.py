@@ -110,6 +110,17 @@ def test_verify_more_units_than_sms(oracle, T):
         out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
                                          float(w.scale), status=dw.status)
         assert_close(bf16_to_f64(out), ref, what=f"verify, {B * 8} units, T={T}, launch {rep}")
+    # split calls: units are (sequence, chunk, kv head, row block); partials merged by the reduce launch
+    for chunk in (64, 208, 512):
+        mc = pda.max_chunks(int(lens.max()), chunk)
+        po = torch.full((B, T, 32, mc, 128), float("nan"), dtype=torch.float32, device="cuda")
+        pl = torch.full((B, T, 32, mc), float("nan"), dtype=torch.float32, device="cuda")
+        for flags in (0, pda.PDA_FLAG_MQ_ONE_UNIT):
+            po.fill_(float("nan"))
+            out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                             float(w.scale), chunk_tokens=chunk, part_o=po, part_lse=pl,
+                                             flags=flags, status=dw.status)
+            assert_close(bf16_to_f64(out), ref, what=f"verify split {chunk}, T={T}, flags {flags}")
     assert int(dw.status.item()) == 0
 
 
