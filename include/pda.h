@@ -18,9 +18,21 @@
  *
  * Conventions
  *   - All data pointers are DEVICE pointers unless a comment says "host".
- *   - The caller owns every buffer. The library allocates no device memory and
- *     keeps no state between calls (TMA descriptors are rebuilt per call on
- *     the host and passed by value).
+ *   - The caller owns every data buffer: inputs, outputs, partials, workspaces,
+ *     status words. TMA descriptors are rebuilt per call on the host and passed by
+ *     value. What the library itself owns, per process, is small and listed here:
+ *       * per device, a second stream and two events, created by the first
+ *         paged_prefix_decode_attention call on that device that is not inside a
+ *         stream capture (the cascade's suffix launch runs on it);
+ *       * per device, 64 claim counters (256 bytes of the library's device image)
+ *         used by the persistent kernel of paged_verify_attention, each left at zero
+ *         by the launch that took it;
+ *       * per device, the PDA_STATIC_SCRATCH_BYTES array of
+ *         paged_decode_attention_static (part of the device image: reserved when the
+ *         image is loaded on that device, see there);
+ *       * one host-side integer, the threshold of pda_set_persistent_threshold.
+ *     No call allocates device memory with cudaMalloc or frees any; nothing else
+ *     is kept between calls.
  *   - Every call enqueues work on `stream` (a cudaStream_t passed as void*) and
  *     returns without synchronising. Nothing reads seq_lens or block_table back
  *     to the host, so a step can be captured in a CUDA graph.
@@ -226,13 +238,11 @@ int kv_append_tokens_fp8(const void* k_new, const void* v_new, void* k_cache, vo
  * taken in turn by the launches and left at zero by each): up to 64 such launches
  * may be in flight at once on a device; a launch captured in a CUDA graph keeps its
  * counter, so one graph must not run beside itself on two streams.
- * e4m3 on tcgen05: the products are e4m3 x e4m3 on the cache's bytes; q and the softmax
- * weights enter as two 8-bit parts each (q to 2^-8, a weight to 2^-7 relative), the
- * page scales through the softmax. An output element is within about 0.3 % of the
- * largest magnitude in its row of the exact result, which meets 2e-2 + 2e-2 |ref| for
- * values of order one; where the dequantised values are far larger, or a tighter
- * bound is wanted, use PDA_FLAG_MQ_MMA_SYNC (weights in f16). Scales must be finite
- * and non-negative (kv_append_fp8 writes them so). */
+ * e4m3 on tcgen05: the products are e4m3 x e4m3 on the cache's bytes; q enters as two
+ * e4m3 parts (exact for every element within 2^-9 of its row's largest) and the softmax
+ * weights as three 8-bit parts that add up to the weight rounded to fp16, the same
+ * precision the mma.sync kernel gives them; the page scales go through the softmax.
+ * Scales must be finite and non-negative (kv_append_fp8 writes them so). */
 int paged_verify_attention(const void* q, const void* k_cache, const void* v_cache,
                            const pda_cache_desc* desc, const float* k_scale,
                            const float* v_scale, const int32_t* block_table,
@@ -366,8 +376,19 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
  * paged_decode_attention(chunk_tokens > 0) followed by paged_decode_reduce does,
  * but keeps part_o / part_lse in a fixed array of PDA_STATIC_SCRATCH_BYTES
  * compiled into the library's device image. It calls no cudaMalloc, cudaFree or
- * other allocating routine. Every process that loads the library holds that
- * array on each GPU it uses, until it exits.
+ * other allocating routine.
+ *
+ * The array is part of the device code of the library, and the CUDA runtime loads
+ * device code lazily: the image that holds the array is loaded on a device -- and
+ * its PDA_STATIC_SCRATCH_BYTES of device memory reserved there, until the process
+ * exits -- by the FIRST call of this function on that device, which looks up the
+ * array's device address (with that device current) and caches it. That first
+ * call therefore synchronises like any module load and fails with the runtime's
+ * out-of-memory code (a positive return value) if the device has no room left.
+ * Make it once per device at start-up: before the process hands the rest of HBM
+ * to its pools, and outside any stream capture (a call with batch 0 is enough and
+ * enqueues nothing). Every later call on that device reserves nothing: the free
+ * memory the runtime reports is the same before and after it.
  *
  * Arguments are those of paged_decode_attention without the partial buffers and
  * flags; `out` is [batch, num_q_heads, head_dim] bf16. The sizes must satisfy
@@ -375,13 +396,11 @@ int paged_decode_step_host(const void* q_host, const void* k_new_host, const voi
  *     + batch*num_q_heads*max_chunks*4  <=  PDA_STATIC_SCRATCH_BYTES,
  * otherwise PDA_ERR_TOO_LARGE is returned and nothing is enqueued.
  *
- * The first call on each device looks up the array's device address (with that
- * device current) and caches it; make that first call outside any stream
- * capture. The array is shared by all calls and keeps the previous call's
- * contents: nothing in it needs to start at zero (attention writes every entry
- * that reduce reads), but two calls whose kernels can overlap on the GPU (different
- * streams, or different host threads without ordering) race on it. Calls on one
- * stream are ordered and safe. */
+ * The array is shared by all calls and keeps the previous call's contents:
+ * nothing in it needs to start at zero (attention writes every entry that reduce
+ * reads), but two calls whose kernels can overlap on the GPU (different streams,
+ * or different host threads without ordering) race on it. Calls on one stream are
+ * ordered and safe. */
 #define PDA_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
 int paged_decode_attention_static(const void* q, const void* k_cache, const void* v_cache,
                                   const pda_cache_desc* desc, const float* k_scale,
@@ -394,6 +413,31 @@ int paged_decode_attention_static(const void* q, const void* k_cache, const void
 /* Diagnostic: decodes all 256 e4m3 bytes with the device decoder the generic
  * kernel uses; out256: device float[256]. */
 int pda_debug_e4m3_decode(float* out256, pda_stream_t stream);
+
+/* Diagnostic: makes the kernels' bounded waits run out. (No counterpart in the
+ * paper; this exercises the library's own failure handling.) Every wait inside the
+ * attention kernels is a wait of a warp on an mbarrier of its own CTA with a poll
+ * limit, after which the kernel records PDA_DEV_TIMEOUT in *status, zero-fills the
+ * unit's output and returns. This call launches one warp that initialises such a
+ * barrier, never arrives at it, and runs the same two wait helpers (the suspended
+ * try_wait form of the TMA rings, the spinning test_wait form of the tensor-core
+ * hand-offs) with `polls` as their limit instead of the built-in 2^20 and 2^24.
+ * Nothing faults and nothing waits without a limit; the context stays usable.
+ *   polls   1 .. 2^20
+ *   status  device int32: receives atomicMax(PDA_DEV_TIMEOUT)
+ *   result  device uint64[3] or NULL: nanoseconds spent in the suspended and in the
+ *           spinning wait, and a mask of the waits that wrongly reported completion
+ *           (must be 0). */
+int pda_debug_wait_timeout(uint32_t polls, int32_t* status, uint64_t* result, pda_stream_t stream);
+
+/* Diagnostic: read-only streaming probe. Reads `bytes` (a multiple of 16) from the
+ * 16-byte aligned device buffer `buf` once with 16-byte loads from 8 CTAs per SM
+ * and writes nothing but (practically never) one counter word `sink` (device
+ * uint32). Timed by the caller with events, bytes / time is the bandwidth a kernel
+ * that only reads HBM can reach on this device: the ceiling beside which the
+ * decode kernels' GB/s are to be read (a copy moves half its bytes as writes and
+ * is the lower figure). */
+int pda_debug_read_probe(const void* buf, uint64_t bytes, uint32_t* sink, pda_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -26,7 +26,7 @@ EXPORTS = ["pda_version", "pda_status_string", "pda_max_chunks", "kv_append",
            "pda_debug_e4m3_decode", "paged_decode_attention_static", "pda_workspace_ints",
            "paged_decode_step", "pda_advance_seq_lens", "paged_window_decode_attention", "kv_append_tokens",
            "paged_verify_attention", "paged_prefix_decode_attention", "kv_append_fp8", "kv_append_tokens_fp8",
-           "pda_set_persistent_threshold"]
+           "pda_set_persistent_threshold", "pda_debug_wait_timeout", "pda_debug_read_probe"]
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
@@ -74,6 +74,8 @@ def lib():
         L.paged_decode_step.argtypes = [vp, vp, vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32, f32,
                                         i32, vp, vp, vp, i32, vp, vp, vp]
         L.pda_debug_e4m3_decode.argtypes = [vp, vp]
+        L.pda_debug_wait_timeout.argtypes = [u32, vp, vp, vp]
+        L.pda_debug_read_probe.argtypes = [vp, C.c_uint64, vp, vp]
         L.paged_decode_attention_static.argtypes = [vp, vp, vp, dp, vp, vp, vp, i32, vp, i32, i32,
                                                     f32, i32, i32, vp, vp, vp]
         _lib = L
@@ -266,6 +268,20 @@ def paged_decode_attention_static(q, k_cache, v_cache, block_table, seq_lens, sc
         chunk_tokens, max_chunks, _ptr(out), _ptr(status), _stream(stream))
     _check(rc, "paged_decode_attention_static")
     return out
+
+
+def debug_wait_timeout(polls, status, result=None, stream=None):
+    """Runs the kernels' two bounded waits on a barrier nobody arrives at, with ``polls`` as the limit;
+    ``status`` (int32[1]) receives PDA_DEV_TIMEOUT, ``result`` (int64[3]) the two durations in ns and the
+    mask of waits that wrongly reported completion."""
+    _check(lib().pda_debug_wait_timeout(int(polls), _ptr(status), _ptr(result), _stream(stream)),
+           "pda_debug_wait_timeout")
+
+
+def debug_read_probe(buf, sink, stream=None):
+    """Enqueues one read-only pass over ``buf`` (any dtype, contiguous, a multiple of 16 bytes)."""
+    nbytes = buf.numel() * buf.element_size()
+    _check(lib().pda_debug_read_probe(_ptr(buf), nbytes, _ptr(sink), _stream(stream)), "pda_debug_read_probe")
 
 
 def advance_seq_lens(seq_lens, delta=1, stream=None):

@@ -94,19 +94,30 @@ int check_attention(const void* q, const void* k_cache, const void* v_cache,
 namespace {
 // A library-owned second stream for the one place where two independent launches of a call can share
 // the GPU (the shared-prefix cascade: its prefix launch leaves SMs idle that the suffix launch can use).
-// Fork and join go through events, so the pattern is also valid inside a stream capture. Created on the
-// first call that is not being captured (creating a stream during a capture is not allowed in every
-// capture mode); until then such calls run their launches one after the other. One process drives one
-// device here, so there is one of these.
+// Fork and join go through events, so the pattern is also valid inside a stream capture. One set per
+// device, created by the first call on that device that is not being captured (creating a stream during
+// a capture is not allowed in every capture mode); until then such calls run their launches one after
+// the other, as they do on a device beyond kMaxDevices.
 struct SideStream {
   std::mutex mu;
   cudaStream_t stream = nullptr;
   cudaEvent_t fork = nullptr, join = nullptr;
 };
-SideStream g_side;
+constexpr int kMaxDevices = 64;
+SideStream g_side[kMaxDevices];
 
-bool side_stream_ready(cudaStream_t main_stream) {  // g_side.mu held
-  if (g_side.stream) return true;
+// The current device's set, or nullptr when there is none to use.
+SideStream* side_stream_of_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return dev >= 0 && dev < kMaxDevices ? &g_side[dev] : nullptr;
+}
+
+bool side_stream_ready(SideStream& side, cudaStream_t main_stream) {  // side.mu held, side's device current
+  if (side.stream) return true;
   cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(main_stream, &st) != cudaSuccess || st != cudaStreamCaptureStatusNone) {
     cudaGetLastError();
@@ -123,9 +134,9 @@ bool side_stream_ready(cudaStream_t main_stream) {  // g_side.mu held
     if (ns) cudaStreamDestroy(ns);
     return false;
   }
-  g_side.stream = ns;
-  g_side.fork = a;
-  g_side.join = b;
+  side.stream = ns;
+  side.fork = a;
+  side.join = b;
   return true;
 }
 
@@ -353,40 +364,40 @@ int paged_prefix_decode_attention(const void* q, const void* k_cache, const void
   p.scale = scale;
   p.out = static_cast<__nv_bfloat16*>(out);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-
-  // The suffix launch (2) is independent of the prefix launch (1) and small, and (1) rarely fills the
-  // GPU (one CTA per SM, chunks x kv heads of them), so (2) runs beside it on the library's second
-  // stream: the fork event is recorded before (1), (1) is submitted first so that its CTAs are placed
-  // first, and (2) is joined before the merge.
-  std::lock_guard<std::mutex> lock(g_side.mu);
-  bool forked = side_stream_ready(s) && cudaEventRecord(g_side.fork, s) == cudaSuccess;
-  if (!forked) cudaGetLastError();
-
   // (1) the shared prefix once: the batch's queries as one block of rows per kv head
   AttnParams pp = p;
   pp.batch = 1;
   pp.chunk_tokens = prefix_chunk_tokens;
   pp.chunk_slot0 = 0;
   pda::MqParams mp{pp, batch, 0, prefix_tokens, prefix_chunks};
-  if (!pda::attention_tma_supports(p)) return PDA_ERR_UNSUPPORTED;
-  if (!(flags & PDA_FLAG_MQ_MMA_SYNC) && pda::attention_mq_tc_supports(mp)) {
-    if (cudaError_t e = pda::launch_attention_mq_tc(mp, s)) return static_cast<int>(e);
-  } else {
-    if (!pda::attention_mq_supports(mp)) return PDA_ERR_UNSUPPORTED;
-    if (cudaError_t e = pda::launch_attention_mq(mp, s)) return static_cast<int>(e);
-  }
+  const bool prefix_tc = !(flags & PDA_FLAG_MQ_MMA_SYNC) && pda::attention_mq_tc_supports(mp);
+  if (!pda::attention_tma_supports(p) || (!prefix_tc && !pda::attention_mq_supports(mp)))
+    return PDA_ERR_UNSUPPORTED;  // (decided before anything is enqueued)
+
+  // The suffix launch (2) is independent of the prefix launch (1) and small, and (1) rarely fills the
+  // GPU (one CTA per SM, chunks x kv heads of them), so (2) runs beside it on the library's second
+  // stream: the fork event is recorded before (1), (1) is submitted first so that its CTAs are placed
+  // first, and (2) is joined before the merge.
+  static std::mutex no_side_mu;  // (a device without a set: nothing to guard, the launches stay on `stream`)
+  SideStream* side = side_stream_of_current_device();
+  std::lock_guard<std::mutex> lock(side ? side->mu : no_side_mu);
+  bool forked = side && side_stream_ready(*side, s) && cudaEventRecord(side->fork, s) == cudaSuccess;
+  if (!forked) cudaGetLastError();
+
+  if (cudaError_t e = prefix_tc ? pda::launch_attention_mq_tc(mp, s) : pda::launch_attention_mq(mp, s))
+    return static_cast<int>(e);
   // (2) every sequence's own suffix, chunk slots after the prefix's
   AttnParams ps = p;
   ps.first_token = prefix_tokens;
   ps.chunk_slot0 = prefix_chunks;
-  if (forked && cudaStreamWaitEvent(g_side.stream, g_side.fork, 0) != cudaSuccess) {
+  if (forked && cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess) {
     cudaGetLastError();
     forked = false;
   }
-  cudaError_t e2 = pda::launch_attention_tma(ps, forked ? g_side.stream : s);
+  cudaError_t e2 = pda::launch_attention_tma(ps, forked ? side->stream : s);
   if (forked) {  // join in any case: a capture must not be left with an open branch
-    cudaError_t ej = cudaEventRecord(g_side.join, g_side.stream);
-    if (ej == cudaSuccess) ej = cudaStreamWaitEvent(s, g_side.join, 0);
+    cudaError_t ej = cudaEventRecord(side->join, side->stream);
+    if (ej == cudaSuccess) ej = cudaStreamWaitEvent(s, side->join, 0);
     if (e2 == cudaSuccess) e2 = ej;
   }
   if (e2 != cudaSuccess) return static_cast<int>(e2);
@@ -539,6 +550,19 @@ int pda_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t delta, pda_st
 int pda_debug_e4m3_decode(float* out256, pda_stream_t stream) {
   if (!out256) return PDA_ERR_INVALID_ARG;
   return static_cast<int>(pda::launch_e4m3_decode(out256, static_cast<cudaStream_t>(stream)));
+}
+
+int pda_debug_wait_timeout(uint32_t polls, int32_t* status, uint64_t* result, pda_stream_t stream) {
+  if (!status || polls == 0 || polls > (1u << 20)) return PDA_ERR_INVALID_ARG;
+  if (result && (reinterpret_cast<uintptr_t>(result) & 7u)) return PDA_ERR_MISALIGNED;
+  return static_cast<int>(pda::launch_wait_timeout(polls, status, result, static_cast<cudaStream_t>(stream)));
+}
+
+int pda_debug_read_probe(const void* buf, uint64_t bytes, uint32_t* sink, pda_stream_t stream) {
+  if (!buf || !sink || bytes == 0 || bytes % 16 != 0) return PDA_ERR_INVALID_ARG;
+  if (!aligned16(buf)) return PDA_ERR_MISALIGNED;
+  return static_cast<int>(pda::launch_read_probe(buf, static_cast<size_t>(bytes), sink,
+                                                 static_cast<cudaStream_t>(stream)));
 }
 
 }  // extern "C"

@@ -124,5 +124,7 @@ cudaError_t launch_kv_append_tokens(const void* k_new, const void* v_new, void* 
                                     const int32_t* seq_lens, int32_t batch, int32_t n_new,
                                     int32_t* status, cudaStream_t stream);
 cudaError_t launch_e4m3_decode(float* out256, cudaStream_t stream);
+cudaError_t launch_wait_timeout(uint32_t polls, int32_t* status, uint64_t* result, cudaStream_t stream);
+cudaError_t launch_read_probe(const void* buf, size_t bytes, uint32_t* sink, cudaStream_t stream);
 
 }  // namespace pda

@@ -63,7 +63,7 @@ reduce_kernel(const float* __restrict__ part_o, const float* __restrict__ part_l
       }
     }
     for (int c = kReduceMaxBlocks * 32; c < n_chunks; ++c) {  // (more than 256 chunks: weights recomputed)
-      const float w = __expf(lse[c] - M);
+      const float w = M > -INFINITY ? __expf(lse[c] - M) : 0.f;  // (every chunk empty: zeros, as above)
       if (v < vecs) {
         const float4 x = __ldg(po + static_cast<int64_t>(c) * vecs + v);
         acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y);

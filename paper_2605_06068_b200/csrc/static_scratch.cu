@@ -9,8 +9,10 @@ namespace {
 
 constexpr size_t kScratchBytes = PDA_STATIC_SCRATCH_BYTES;
 
-// Scratch for the split-KV partials. File-scope device storage: every device
-// that loads this library carries these bytes until the process exits.
+// Scratch for the split-KV partials. File-scope device storage: a device carries
+// these bytes from the moment this file's device image is loaded on it (the
+// runtime loads images lazily, so that is the first address lookup below) until
+// the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
@@ -19,7 +21,9 @@ void* g_scratch_ptr[kMaxDevices] = {};
 
 // Device address of g_static_scratch on the current device. In host code the
 // symbol's name is only a handle, so the address is looked up once per device
-// (with that device current) and cached.
+// (with that device current) and cached. The first lookup on a device loads the
+// image and can fail (no room left for the array): the error is returned, and
+// nothing is cached, so a later call tries again.
 cudaError_t scratch_address(void** out) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -52,9 +56,11 @@ extern "C" int paged_decode_attention_static(
   const size_t o_bytes = (rows * desc->head_dim * 4 + 255) & ~static_cast<size_t>(255);
   const size_t need = o_bytes + rows * 4;
   if (need > kScratchBytes) return PDA_ERR_TOO_LARGE;
-  if (batch == 0) return PDA_OK;
+  // (before the empty-batch return: a start-up call with batch 0 is how a caller gets the image that holds
+  // the array loaded, and its bytes reserved, while the device still has room)
   void* base = nullptr;
   if (cudaError_t e = scratch_address(&base)) return static_cast<int>(e);
+  if (batch == 0) return PDA_OK;
   float* part_o = static_cast<float*>(base);
   float* part_lse = reinterpret_cast<float*>(static_cast<unsigned char*>(base) + o_bytes);
   if (int rc = paged_decode_attention(q, k_cache, v_cache, desc, k_scale, v_scale, block_table,

@@ -10,9 +10,11 @@ namespace pda {
 constexpr int kUmmaRows = 128;  // UMMA M: query rows per CTA, one TMEM lane each
 
 // Spinning bounded wait (no suspension): the waits on the MMA/softmax hand-off are short and on the
-// critical path, where the wake-up latency of a suspended try_wait shows.
-__device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < (1u << 24); ++i)
+// critical path, where the wake-up latency of a suspended try_wait shows. A poll is a test_wait and its
+// loop overhead, some tens of clocks: 2^24 of them give up after a few tenths of a second.
+constexpr uint32_t kTestSpinLimit = 1u << 24;
+__device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kTestSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_test_wait(bar, parity)) return true;
   return false;
 }

@@ -9,8 +9,9 @@
 
 namespace pda {
 
-// A bounded mbarrier wait polls try_wait at most kSpinLimit times, each poll suspended for at
-// most kSuspendNs: it gives up after roughly a second instead of hanging.
+// A bounded mbarrier wait polls try_wait at most kSpinLimit times, each poll suspended by the hardware
+// for at most kSuspendNs: it gives up after about one second (2^20 x 1 us) instead of hanging.
+// pda_debug_wait_timeout runs these helpers on a barrier nobody arrives at and reports what a poll costs.
 constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr uint32_t kSuspendNs = 1000;
 
@@ -42,9 +43,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kSpinLimit polls.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
+// Bounded wait: false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }

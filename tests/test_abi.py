@@ -133,3 +133,13 @@ def test_new_entry_points_validate_without_a_gpu(lib):
     # the allocation-free entry point rejects oversize problems before touching the device
     assert lib.paged_decode_attention_static(P, P, P, C.byref(d), None, None, P, 4, P, 64, 32, 0.1, 16,
                                              4096, P, None, None) == -4
+
+
+def test_diagnostic_calls_check_their_arguments_without_a_gpu(lib):
+    assert lib.pda_debug_wait_timeout(0, 0x1000, None, None) == -1
+    assert lib.pda_debug_wait_timeout((1 << 20) + 1, 0x1000, None, None) == -1
+    assert lib.pda_debug_wait_timeout(100, None, None, None) == -1
+    assert lib.pda_debug_wait_timeout(100, 0x1000, 0x2004, None) == -3
+    assert lib.pda_debug_read_probe(None, 1 << 20, 0x1000, None) == -1
+    assert lib.pda_debug_read_probe(0x1000, 24, 0x2000, None) == -1
+    assert lib.pda_debug_read_probe(0x1008, 32, 0x2000, None) == -3

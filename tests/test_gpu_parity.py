@@ -462,11 +462,16 @@ def test_reduce_many_chunks_and_widths(oracle, D, Cm):
         pl[b, :, n:] = np.nan
     pl[0, 1, 0] = -np.inf                   # an empty chunk inside the range: weight 0
     po[0, 1, 0] = 0.0
+    # a row whose chunks are ALL empty (what a unit skipped for a bad length leaves behind): zeros, also
+    # where the weights are recomputed beyond the register-held blocks
+    pl[1, 2, :] = -np.inf
+    po[1, 2, :] = 0.0
     ref, _ = oracle.paged_decode_reduce(po.astype(np.float64), pl.astype(np.float64), seq, chunk)
     out = pda.paged_decode_reduce(torch.from_numpy(po).cuda(), torch.from_numpy(pl).cuda(),
                                   torch.from_numpy(seq).cuda(), chunk)
     assert_close(bf16_to_f64(out), ref, what=f"reduce Cm={Cm} D={D}", norm=False)
     assert (bf16_to_f64(out)[4] == 0).all()
+    assert (bf16_to_f64(out)[1, 2] == 0).all() and (ref[1, 2] == 0).all()
 
 
 # ---- the end-to-end host call ---------------------------------------------------------------
