@@ -27,7 +27,7 @@
 // issued from inside a divergent branch, a TMA copy or an MMA cost 90-200 clocks each here and the
 // issuing thread was the bottleneck; this way they cost 25-35. S and P are double-buffered:
 //   S warp:     S(j) as soon as stage j has landed and softmax(j-2) has loaded S(j-2) into registers
-//               (bar_sfree) -> commit(bar_s[j&1])
+//               (bar_sfree; e4m3: P(j-3) . V has completed, bar_buf) -> commit(bar_s[j&1])
 //   PV warp:    wait bar_p[i&1] -> PV(i), l(i) -> commit(stage empty), commit(bar_pv[i&1])
 //   softmax:    wait bar_s[i&1] -> tcgen05.ld S -> arrive(bar_sfree) -> mask (boundary tiles), row max
 //               of the raw scores -> running max of iteration i-1 from the other set (bar_m, shared
@@ -40,9 +40,14 @@
 // more MMA per part into the same accumulator:
 //   Q = hi + lo, both e4m3, after a per-row power of two that brings the row's largest magnitude into
 //       [128, 256) (it goes into the row's score constant): 2 x 4 MMAs M128 x N64 x K32 per iteration
-//   P = hi (e4m3, round to nearest) + lo (e5m2: its exponent range keeps weights far below the row's
-//       largest one, where e4m3 stops at 2^-9): 2 x 2 MMAs M128 x N128 x K32, a step spanning two pages
-//       whose V tiles are contiguous; |p - hi - lo| <= max(2^-7 p, 2^-17)
+//   P = hi (e4m3) + mid (e4m3) + lo (e5m2), each the rounded remainder of the one before: together they
+//       are the weight rounded to f16, exactly, for weights down to 2^-6 (the reference maximum is kept
+//       2^4 below the row's largest score, so that is 2^-10 of the largest weight); 3 x 2 MMAs
+//       M128 x N128 x K32, a step spanning two pages whose V tiles are contiguous. Two parts (2^-7
+//       relative) were not enough: with page scales spread over many powers of two an output element
+//       could miss 2e-2 + 2e-2 |ref| by cancellation.
+//   S(it) and P(it) share one of three 64-column buffers (it % 3): P is written over the scores it came
+//       from, and S(it + 3) follows once P(it) . V has completed (bar_buf).
 // The page scales stay out of the tiles: the K scale is the score factor of the page's 16 columns; the V
 // scale enters as log2(v_scale) added to the score, so that P carries it into P . V_raw, and each page's
 // sum of P divided by v_scale is its share of the row sum, which the softmax warps keep in registers.
@@ -92,14 +97,20 @@ constexpr uint32_t kTcRegsSoftmax = 208, kTcRegsControl = 72;
 // Tensor memory columns (32-bit each, 128 lanes = query rows), bf16: S buffers 0..63 and 64..127 (f32),
 // O 128..255 (f32), Q 256..319 (bf16 pairs along d), P buffers 320..351 and 352..383 (bf16 pairs along
 // tokens), l 384..399. Allocations are powers of two.
-// e4m3: S as above; each softmax set accumulates into an O of its own (128..255 and 256..383); Q 384..447
-// (four elements to a column: 32 columns of high parts, then 32 of low parts); P buffers 448..479 and
-// 480..511 (four tokens to a column: 16 columns of high parts, then 16 of low parts).
+// e4m3: three S / P buffers 0..63, 64..127, 128..191 (iteration it uses it % 3: S as 64 f32 columns, then P
+// over it, four tokens to a column: 16 columns each of high, middle and low parts); each softmax set
+// accumulates into an O of its own (192..319 and 320..447); Q 448..511 (four elements to a column: 32
+// columns of high parts, then 32 of low parts).
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kTmemO = 128, kTmemL = 384;  // l (bf16): row sums of P, 16 columns (all equal)
-template <bool kFp8> constexpr uint32_t kTmemQ = kFp8 ? 384 : 256;
-template <bool kFp8> constexpr uint32_t kTmemP = kFp8 ? 448 : 320;
+constexpr uint32_t kTmemL = 384;  // l (bf16): row sums of P, 16 columns (all equal)
+template <bool kFp8> constexpr uint32_t kTmemO = kFp8 ? 192 : 128;
+template <bool kFp8> constexpr uint32_t kTmemQ = kFp8 ? 448 : 256;
+constexpr uint32_t kTmemPBf16 = 320;
+constexpr int kFp8Bufs = 3;
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the max grows this much
+// e4m3: the reference is set this far below the largest score seen (log2 units), so that the weights start
+// at 2^4 and may grow to 2^8 before a rescale: the three 8-bit parts of a weight are exact from 2^-6 up.
+constexpr float kFp8RefBelowMax = 4.f;
 
 template <int D, bool kFp8>
 __global__ void __launch_bounds__((TcCfg<D, kFp8>::kThreads), 1)
@@ -117,9 +128,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   float* rowc_sh = m_sh + 2 * kTcRows;                                     // e4m3: [128] score constant of the row
   float* l_sh = rowc_sh + kTcRows;                                         // e4m3: [2][128] the sets' row sums
   float* scale_sh = l_sh + 2 * kTcRows;                                    // e4m3: [stage][4 c, 4 a, 4 1/v, 4 unused]
-  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2][4]
+  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2][4], buf[3] (+1 unused)
   uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes + kTcRowBytes + C::kScaleBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 16);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 20);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
   int* rank_slot = cta_err + 1;
 
@@ -149,6 +160,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kTcStages;
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
   const uint32_t bar_sfree = bar_pv + 16, bar_m = bar_sfree + 16;
+  const uint32_t bar_buf = bar_m + 64;  // e4m3: S / P buffer k is free again (its P . V has completed)
   if constexpr (!kFp8) {
     for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads)
       reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;  // 1.0 as bf16 pairs
@@ -167,6 +179,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
       for (int w = 0; w < 4; ++w) mbar_init(bar_m + 8 * (4 * k + w), 1);  // per warp: rows w*32.. of set k
     }
+    for (int k = 0; k < kFp8Bufs; ++k) mbar_init(bar_buf + 8 * k, 1);
     *cta_err = 0;
     fence_mbar_init();
     fence_proxy_async();
@@ -217,8 +230,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const int n_iters = (n_pages + kTcPagesPerIter - 1) / kTcPagesPerIter;
 
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTmemO;  // S buffer k at tmem_s + 64 k
-  const uint32_t tmem_q = tmem_base + kTmemQ<kFp8>, tmem_p = tmem_base + kTmemP<kFp8>;  // P buffer k at tmem_p + 32 k
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTmemO<kFp8>;  // S buffer k at tmem_s + 64 k
+  const uint32_t tmem_q = tmem_base + kTmemQ<kFp8>;
+  const uint32_t tmem_p = tmem_base + kTmemPBf16;  // bf16: P buffer k at tmem_p + 32 k (e4m3: P lies over its S)
 
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
 
@@ -369,9 +383,15 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int u_tail0 = __shfl_sync(0xffffffffu, L - page0 * kPageSize, 0);  // tokens from the first page to the end
     bool ok = true;
     uint32_t stage_i = 0, stage_par = 0;  // the iteration's ring stage and the phase parity of its full barrier
+    uint32_t buf_i = 0, buf_round = 0;    // e4m3: it % 3 and it / 3
     for (int it = 0; it < u_iters; ++it) {
-      // S(it) overwrites the buffer of S(it-2): the softmax warps have loaded that into registers
-      if (it >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (it & 1), ((it - 2) >> 1) & 1);
+      if constexpr (kFp8) {
+        // S(it) overwrites the buffer of S(it-3) and P(it-3): P(it-3) . V has completed
+        if (it >= kFp8Bufs) ok = mbar_wait_bounded(bar_buf + 8 * buf_i, (buf_round - 1) & 1);
+      } else {
+        // S(it) overwrites the buffer of S(it-2): the softmax warps have loaded that into registers
+        if (it >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (it & 1), ((it - 2) >> 1) & 1);
+      }
       if (ok) ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);  // the block has landed
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -398,7 +418,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         __syncwarp();
       }
       tc_fence_after();
-      const uint32_t d = u_tmem + 64 * (it & 1);
+      const uint32_t d = u_tmem + 64 * (kFp8 ? buf_i : static_cast<uint32_t>(it & 1));
       // S[:, 0..64) = Q . K^T over the 64 stacked token rows
       // (rows of pages that were not loaded hold stale data: those columns are masked later)
       const uint64_t kd0 = tc_desc(stage, 16, 1024);
@@ -422,6 +442,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       tc_commit_if(leader, bar_s + 8 * (it & 1));
       if (++stage_i == kTcStages) { stage_i = 0; stage_par ^= 1; }
+      if (++buf_i == kFp8Bufs) { buf_i = 0; ++buf_round; }
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   };
@@ -437,6 +458,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int u_pages = __shfl_sync(0xffffffffu, n_pages, 0);
     bool ok = true;
     uint32_t stage_i = 0;  // the iteration's ring stage
+    uint32_t buf_i = 0;    // e4m3: it % 3
     for (int it = 0; it < u_iters; ++it) {
       ok = mbar_wait_bounded(bar_p + 8 * (it & 1), (it >> 1) & 1);
       ok = __all_sync(0xffffffffu, ok);
@@ -444,17 +466,18 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       tc_fence_after();
       const uint32_t stage = ring + stage_i * C::kOperandBytes;
       const int n_here = min(kTcPagesPerIter, u_pages - it * kTcPagesPerIter);
-      const uint32_t pa0 = u_tmem + kTmemP<kFp8> + 32 * (it & 1);
+      const uint32_t pa0 = kFp8 ? u_tmem + 64 * buf_i : u_tmem + kTmemPBf16 + 32 * (it & 1);
       // V read MN-major. LBO: next 64 columns of d (bf16; an e4m3 line holds all 128), SBO: next 8 tokens
       const uint64_t vd0 = tc_desc(stage + kTcKBytes, kPageSize * 128, 1024);
       if constexpr (kFp8) {
         // O[it % 2] += P[:, 32j .. 32j+32) . V : one K = 32 step per two pages (their tiles are contiguous),
-        // once with the high and once with the low parts of P; the row sums are kept by the softmax warps
+        // once with each of the three parts of P (high, middle: e4m3; low: e5m2); the row sums are kept by
+        // the softmax warps
         auto pv_pair = [&](int j) {
 #pragma unroll
-          for (int part = 0; part < 2; ++part)
-            tc_mma_ts_if<true>(leader, u_tmem + kTmemO + D * (it & 1), pa0 + 16 * part + 8 * j,
-                               vd0 + static_cast<uint64_t>(j * (2 * kTcTileBytes / 16)), part ? idesc_pv_lo : idesc_pv,
+          for (int part = 0; part < 3; ++part)
+            tc_mma_ts_if<true>(leader, u_tmem + kTmemO<true> + D * (it & 1), pa0 + 16 * part + 8 * j,
+                               vd0 + static_cast<uint64_t>(j * (2 * kTcTileBytes / 16)), part == 2 ? idesc_pv_lo : idesc_pv,
                                (it > 1 || j > 0 || part > 0) ? 1u : 0u);
         };
         pv_pair(0);
@@ -464,7 +487,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
         // and l += P[:, 16j .. 16j+16) . 1 : the row sums of exactly the P that multiplies V
         auto pv_page = [&](int j) {
           const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-          tc_mma_ts_if<false>(leader, u_tmem + kTmemO, pa0 + 8 * j, vd0 + static_cast<uint64_t>(j * (kTcTileBytes / 16)), idesc_pv, acc);
+          tc_mma_ts_if<false>(leader, u_tmem + kTmemO<false>, pa0 + 8 * j, vd0 + static_cast<uint64_t>(j * (kTcTileBytes / 16)), idesc_pv, acc);
           tc_mma_ts_if<false>(leader, u_tmem + kTmemL, pa0 + 8 * j, ones_desc, idesc_l, acc);
         };
         if (n_here == kTcPagesPerIter) {
@@ -476,7 +499,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       tc_commit_if(leader, empty0 + 8 * stage_i);     // the stage may be refilled once these MMAs have read it
       tc_commit_if(leader, bar_pv + 8 * (it & 1));    // O (and l) updated, P buffer free again
+      if constexpr (kFp8) tc_commit_if(leader, bar_buf + 8 * buf_i);  // ... which the S issue warp waits for
       if (++stage_i == kTcStages) stage_i = 0;
+      if (++buf_i == kFp8Bufs) buf_i = 0;
     }
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   };
@@ -500,6 +525,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     float l_set = 0.f, m_l = -INFINITY, rowc = 0.f;
     if constexpr (kFp8) rowc = rowc_sh[t];
     uint32_t sc_stage = set % kTcStages;  // ring stage of this set's next iteration
+    uint32_t my_buf = set;                 // e4m3: S / P buffer of this set's next iteration (it % 3)
     bool alive = true;
     auto fail = [&]() { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; };
     for (int it = set; it < n_iters; it += 2) {
@@ -509,12 +535,17 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       if (!ok) { fail(); break; }
       tc_fence_after();
       uint32_t sv[2][32];
-      tmem_ld32(tmem_s + 64 * set + lane_base, sv[0]);
-      tmem_ld32(tmem_s + 64 * set + lane_base + 32, sv[1]);
+      const uint32_t sp_buf = tmem_s + 64 * (kFp8 ? my_buf : static_cast<uint32_t>(set)) + lane_base;
+      tmem_ld32(sp_buf, sv[0]);
+      tmem_ld32(sp_buf + 32, sv[1]);
       tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_tc(my_sfree);  // S(it) is in registers: S(it+2) may overwrite its buffer
+      if constexpr (kFp8) {
+        my_buf = my_buf >= 1 ? my_buf - 1 : my_buf + 2;  // (it + 2) % 3
+      } else {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_tc(my_sfree);  // S(it) is in registers: S(it+2) may overwrite its buffer
+      }
       const int tok0 = (page0 + it * kTcPagesPerIter) * kPageSize;
       const int n_vis = min(lim, t1) - tok0;  // visible columns of this row in this iteration (may be <= 0)
       if (__any_sync(0xffffffffu, n_vis < kTcPagesPerIter * kPageSize)) {  // boundary tiles only
@@ -574,7 +605,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       // lazy rescaling: keep the old reference unless the max grew past the threshold
       float m_new = m_ref;
-      if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = fmaxf(m_ref, mx);
+      if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = kFp8 ? mx - kFp8RefBelowMax : fmaxf(m_ref, mx);
       const bool need = m_new != m_ref && m_ref != -INFINITY;
       if constexpr (!kFp8) {
         m_sh[(it & 1) * kTcRows + t] = m_new;
@@ -597,24 +628,26 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
         for (int cb = 0; cb < D / 32 + (kFp8 ? 0 : 1); ++cb) {  // O, then (bf16) the block of columns that holds l
           uint32_t ov[32];
-          tmem_ld32(my_o + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
+          tmem_ld32(my_o + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO<false>), ov);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
-          tmem_st32(my_o + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO), ov);
+          tmem_st32(my_o + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO<false>), ov);
         }
         tmem_wait_st();
       }
       m_ref = m_new;
       const float ref = m_ref == -INFINITY ? 0.f : m_ref;
       uint32_t pw[32];
+      uint32_t pw_lo[kFp8 ? 16 : 1];  // e4m3: the low parts of P
       if constexpr (kFp8) {
         if (m_l != m_ref) {  // this set's row sum follows the reference (changed here or by the other set)
           l_set *= ex2(m_l - m_ref);
           m_l = m_ref;
         }
-        // P = exp2(x - ref) as hi (e4m3) + lo (e5m2), four tokens to a column: columns 0..15 the high
-        // parts, 16..31 the low parts (the A operands of the two P . V products)
+        // P = exp2(x - ref) as hi (e4m3) + mid (e4m3) + lo (e5m2), four tokens to a column: columns 0..15
+        // the high parts, 16..31 the middle parts, 32..47 the low parts (the A operands of the three
+        // P . V products)
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const uint64_t c2 = f32x2(__float_as_uint(cq[q]), __float_as_uint(cq[q]));
@@ -622,7 +655,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
           uint64_t sum2 = 0ull;
 #pragma unroll
           for (int j = 8 * q; j < 8 * q + 8; j += 2) {  // two pairs = four tokens = one column
-            uint32_t hi[2], lo[2];
+            uint32_t hi[2], mid[2], lo[2];
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
               const uint64_t x2 = fma_f32x2(f32x2(sv[j >> 4][(2 * (j + e)) & 31], sv[j >> 4][(2 * (j + e) + 1) & 31]), c2, nr2);
@@ -630,10 +663,11 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
               f32x2_split(x2, x0, x1);
               const float p0 = ex2(x0), p1 = ex2(x1);
               sum2 = add_f32x2(sum2, f32x2(__float_as_uint(p0), __float_as_uint(p1)));
-              split_e4m3_e5m2_x2(p0, p1, hi[e], lo[e]);
+              split_e4m3_e4m3_e5m2_x2(p0, p1, hi[e], mid[e], lo[e]);
             }
             pw[j >> 1] = hi[0] | (hi[1] << 16);
-            pw[16 + (j >> 1)] = lo[0] | (lo[1] << 16);
+            pw[16 + (j >> 1)] = mid[0] | (mid[1] << 16);
+            pw_lo[j >> 1] = lo[0] | (lo[1] << 16);
           }
           float s0, s1;
           f32x2_split(sum2, s0, s1);
@@ -652,12 +686,20 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
           pw[j] = pack2<false>(ex2(x0), ex2(x1));
         }
       }
-      if (it >= 2) {  // PV(it-2) has finished reading the P buffer this iteration writes
+      if (it >= 2) {
+        // bf16: PV(it-2) has finished reading the P buffer this iteration writes. (e4m3: P goes over its own
+        // S; the wait keeps this set's view of the barrier one phase behind at most, which the parity
+        // waits on it rely on)
         ok = mbar_spin_bounded(my_pv, (k - 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
       }
-      tmem_st32(tmem_p + 32 * set + lane_base, pw);
+      if constexpr (kFp8) {
+        tmem_st32(sp_buf, pw);
+        tmem_st16(sp_buf + 32, pw_lo);
+      } else {
+        tmem_st32(tmem_p + 32 * set + lane_base, pw);
+      }
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();

@@ -76,19 +76,25 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
   asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
   return r;
 }
-// x = hi + lo, hi in e4m3 (x rounded to nearest), lo in e5m2 (the remainder, rounded): two bytes of each
-// for two values, 0 <= x <= 448. |x - hi - lo| <= max(2^-7 |x|, 2^-17): the wider exponent range of e5m2
-// keeps the weights far below the row's largest one (e4m3 alone stops at 2^-9) to three significant bits.
-// The remainder is taken in f16 pairs, where it is exact.
-__device__ __forceinline__ void split_e4m3_e5m2_x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+// x = hi + mid + lo for two values 0 <= x <= 448: hi = e4m3(x), mid = e4m3(x - hi), lo = e5m2(x - hi - mid),
+// each rounded to nearest, two bytes of each part. x is first rounded to f16 and the remainders are taken
+// in f16 pairs, where they are exact; hi keeps the top four significant bits, mid the next four, and what
+// is left (at most three) fits e5m2: the three parts add up to f16(x) exactly as long as no part falls
+// below its format's range, i.e. for x >= 2^-6. Below that e4m3's subnormal step of 2^-9 takes bits from
+// hi and mid and the sum is within 2^-7 x, never worse than 2^-17.
+__device__ __forceinline__ void split_e4m3_e4m3_e5m2_x2(float x0, float x1, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
   uint32_t xh, back;
-  uint16_t h, l;
+  uint16_t h, m, l;
   asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(xh) : "f"(x1), "f"(x0));
   asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(h) : "r"(xh));
   asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(h));
   asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(xh) : "r"(xh), "r"(back));
+  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(m) : "r"(xh));
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(m));
+  asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(xh) : "r"(xh), "r"(back));
   asm("cvt.rn.satfinite.e5m2x2.f16x2 %0, %1;" : "=h"(l) : "r"(xh));
   hi = h;
+  mid = m;
   lo = l;
 }
 

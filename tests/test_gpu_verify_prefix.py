@@ -199,9 +199,9 @@ def test_verify_fp8_under_unequal_scales(oracle, flags, spread):
     the score factor and the V scale into the exponent and divides it out of the row sum), pages with a
     zero scale, query rows of very different magnitude (Q is split into two e4m3 parts after a per-row
     power-of-two scaling), and a lone dominant key (P = 1 next to tiny weights).
-    moderate: V scales within 2^-3 .. 2^3 of each other, checked with the element-wise tolerance.
-    extreme: V scales over 2^-12 .. 2^8, values in the hundreds: the weights P reach the tensor core as
-    e4m3 + e5m2 pairs (2^-7 relative), so the bound is relative to the row's largest output, 1 %."""
+    moderate: V scales within 2^-3 .. 2^3 of each other; extreme: V scales over 2^-12 .. 2^8, values in
+    the hundreds, where an output element can be small by cancellation between large terms. Both are
+    checked element by element against the stated e4m3 tolerance, on every kernel choice."""
     rng = np.random.default_rng(77)
     lens = [1000, 333, 64, 17]
     T = 8
@@ -227,13 +227,7 @@ def test_verify_fp8_under_unequal_scales(oracle, flags, spread):
                                      float(w.scale), k_scale=torch.from_numpy(ks).cuda(),
                                      v_scale=torch.from_numpy(vs).cuda(), flags=flags, status=dw.status)
     got = bf16_to_f64(out)
-    if spread == "moderate":
-        assert_close(got, ref, "e4m3", what=f"fp8 unequal scales flags {flags}")
-    else:
-        assert np.isfinite(got).all()
-        row_max = np.abs(ref).max(axis=-1, keepdims=True)
-        worst = (np.abs(got - ref) / (2e-2 + 1e-2 * row_max)).max()
-        assert worst <= 1.0, f"fp8 extreme scales flags {flags}: max err / (2e-2 + 1% of row max) = {worst:.3f}"
+    assert_close(got, ref, "e4m3", what=f"fp8 unequal scales ({spread}) flags {flags}")
     # the dominant key's row is that value row (times its scale), to the rounding of the output
     vrow = dec[w.v_cache[page, g, slot]] * float(vs[page, g])
     assert np.abs(got[0, T - 1, 5] - vrow).max() <= 2e-2 + 2e-2 * np.abs(vrow).max()

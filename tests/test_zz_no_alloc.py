@@ -78,7 +78,7 @@ def test_static_scratch_reserves_nothing_after_its_first_call():
     mc = pda.max_chunks(1300, 128)
     # the start-up call: an empty batch is enough and enqueues nothing
     pda.paged_decode_attention_static(dw.q[:0], dw.k_cache, dw.v_cache, dw.block_table[:0], dw.seq_lens[:0],
-                                      float(w.scale), 128, mc, out=out[:0])
+                                      float(w.scale), 128, mc, out=out)
     # one full call, so that the kernels it launches are loaded too (the runtime loads code on first use)
     pda.paged_decode_attention_static(dw.q, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
                                       float(w.scale), 128, mc, out=out, status=dw.status)
