@@ -347,13 +347,16 @@ int pda_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t delta, pda_st
  * `out` back to out_host; all on `stream`, without synchronising. The KV cache
  * itself stays resident on the device between steps. *_dev are device buffers
  * of the same sizes as their host counterparts.
- * In place: q_dev, k_new_dev, v_new_dev and out_dev may each be NULL; the kernel
- * then reads (for out: writes) the host buffer itself over the bus while it
- * streams the cache, and that copy and its launch drop out of the step. This
- * needs pinned host memory that is mapped into the device's address space
- * (cudaHostAlloc, cudaHostRegister); PDA_ERR_INVALID_ARG otherwise. With
- * out_dev == NULL the result exists in out_host only. block_table and seq_lens
- * are always copied (every CTA reads them). */
+ * In place: q_dev, k_new_dev, v_new_dev, block_table_dev, seq_lens_dev and
+ * out_dev may each be NULL; the kernel then reads (for out: writes) the host
+ * buffer itself over the bus while it streams the cache, and that copy and its
+ * launch drop out of the step. This needs pinned host memory that is mapped into
+ * the device's address space (cudaHostAlloc, cudaHostRegister);
+ * PDA_ERR_INVALID_ARG otherwise. With out_dev == NULL the result exists in
+ * out_host only. Every CTA reads seq_lens and its row of block_table at its
+ * start, so reading those two in place trades two copies ahead of the launch
+ * for a bus round trip inside each CTA's start; the host must not change any
+ * in-place buffer before the step has completed. */
 int paged_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,
                            const int32_t* block_table_host, const int32_t* seq_lens_host,
                            void* q_dev, void* k_new_dev, void* v_new_dev,

@@ -71,6 +71,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
   const int gid = lane >> 2, tq = lane & 3;
   const int c = blockIdx.x, g = blockIdx.y;
   int b = blockIdx.z;
+  int L_ranked = -1;  // the unit's length when the ranking below has it at hand (saves a trip to memory)
   if (p.chunk_tokens == 0 && p.batch <= kMaxLptBatch && p.batch > 1) {
     // unsplit units differ in length by the spread of seq_lens: serve the longest first. The CTA
     // with blockIdx.z = r takes the r-th longest sequence (ties by index), so long units start
@@ -82,10 +83,11 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       const int Lj = lens[j];
       int rank = 0;
       for (int i = 0; i < p.batch; ++i) rank += (lens[i] > Lj) || (lens[i] == Lj && i < j);
-      if (rank == static_cast<int>(blockIdx.z)) cta_err[2] = j;
+      if (rank == static_cast<int>(blockIdx.z)) { cta_err[2] = j; cta_err[3] = Lj; }
     }
     __syncthreads();
     b = cta_err[2];
+    L_ranked = cta_err[3];
     __syncthreads();  // lens aliases the ring: done with it before any copy lands
   }
   const int G = p.group;
@@ -95,7 +97,7 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
   // fused step: this launch also writes `out` (merging split-KV partials through the
   // workspace's per-unit chunk counters) and applies the append
   const bool fuse = sp.fuse_reduce != 0;
-  const int L = max(p.seq_lens[b], 0);
+  const int L = L_ranked >= 0 ? L_ranked : max(p.seq_lens[b], 0);
   int t0 = p.first_token, t1 = L;
   if (split) {
     t0 = p.first_token + c * p.chunk_tokens;

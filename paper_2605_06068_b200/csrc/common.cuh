@@ -96,6 +96,9 @@ cudaError_t launch_kv_append_e4m3(const void* k_new, const void* v_new, void* k_
                                   const int32_t* seq_lens, int32_t batch, int32_t n_new, int32_t* status,
                                   cudaStream_t stream);
 cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t delta, cudaStream_t stream);
+// table_host / lens_host: device addresses of pinned, mapped host memory
+cudaError_t launch_stage_tables(const int32_t* table_host, int32_t* table_dev, int64_t n_table,
+                                const int32_t* lens_host, int32_t* lens_dev, int32_t batch, cudaStream_t stream);
 cudaError_t launch_attention_generic(const AttnParams& p, cudaStream_t stream);
 // Returns cudaErrorNotSupported when the shape is outside the fast kernel's set.
 cudaError_t launch_attention_tma(const AttnParams& p, cudaStream_t stream);

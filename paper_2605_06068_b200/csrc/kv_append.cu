@@ -194,4 +194,24 @@ cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int32_t batch, int32_t de
   return cudaGetLastError();
 }
 
+// Copies the step's block table and sequence lengths from pinned, device-mapped host memory into
+// their device buffers with one launch (a thread per int32, reads coalesced over the bus): two small
+// cudaMemcpyAsync calls ahead of the step cost more than this kernel does.
+__global__ void stage_tables_kernel(const int32_t* __restrict__ table_host, int32_t* __restrict__ table_dev,
+                                    int64_t n_table, const int32_t* __restrict__ lens_host,
+                                    int32_t* __restrict__ lens_dev, int32_t batch) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n_table) table_dev[i] = table_host[i];
+  else if (i - n_table < batch) lens_dev[i - n_table] = lens_host[i - n_table];
+}
+
+cudaError_t launch_stage_tables(const int32_t* table_host, int32_t* table_dev, int64_t n_table,
+                                const int32_t* lens_host, int32_t* lens_dev, int32_t batch, cudaStream_t stream) {
+  const int64_t n = n_table + batch;
+  if (n == 0) return cudaSuccess;
+  stage_tables_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(table_host, table_dev, n_table,
+                                                                               lens_host, lens_dev, batch);
+  return cudaGetLastError();
+}
+
 }  // namespace pda

@@ -514,6 +514,20 @@ def test_step_host_matches_device_calls(oracle):
         assert_close(got2, ref, what=f"step_host in place chunk {chunk}")
         assert (bf16_to_bits(dw.k_cache) == k_ref).all()
         assert int(dw.status.item()) == 0
+        # everything in place: block_table and seq_lens are read from the pinned host buffers too, so
+        # the step is the kernel launch and nothing else
+        dw = DeviceWorkload(w)
+        out_host3 = torch.zeros(w.q.shape, dtype=torch.int16).pin_memory()
+        pda.paged_decode_step_host(hq.view(torch.bfloat16), hk, hv, hbt, hsl, None, None, None, None, None,
+                                   dw.k_cache, dw.v_cache, float(w.scale), chunk, po, pl,
+                                   None, out_host3, workspace=pda.new_workspace(w.batch, 8),
+                                   status=dw.status)
+        torch.cuda.synchronize()
+        got3 = W.bf16_bits_to_f32(out_host3.numpy().view(np.uint16)).astype(np.float64)
+        assert_close(got3, ref, what=f"step_host all in place chunk {chunk}")
+        assert (got3 == got2).all()
+        assert (bf16_to_bits(dw.k_cache) == k_ref).all()
+        assert int(dw.status.item()) == 0
     with pytest.raises(RuntimeError):
         pda.paged_decode_step_host(hq.view(torch.bfloat16), hk, hv, hbt, hsl, None, None, None, dbt, dsl,
                                    dw.k_cache, dw.v_cache, float(w.scale), 0, None, None,
