@@ -401,6 +401,8 @@ def run_workload(name, args, ctx, headline):
     t_end.record(stream)
     barrier()
     ms_b2b = t_start.elapsed_time(t_end) / K
+    if int(status.item()) != 0:
+        raise RuntimeError(f"device status {int(status.item())}: {pda.status_string(int(status.item()))}")
 
     # ---- the same step captured once in a CUDA graph and replayed (no host launch work) ----------------
     ms_graph = 0.0

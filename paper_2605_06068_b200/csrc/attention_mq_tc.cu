@@ -55,6 +55,8 @@
 // like split-KV partials, so the sets exchange nothing per iteration. A twelfth, idle warp completes
 // the third warpgroup so that setmaxnreg can move registers from the control warps to the softmax warps.
 // All mbarrier waits are bounded; TMEM is always released before the CTA exits.
+#include <type_traits>
+
 #include "common.cuh"
 #include "tma_ptx.cuh"
 #include "tcgen05_ptx.cuh"
@@ -128,9 +130,9 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   float* rowc_sh = m_sh + 2 * kTcRows;                                     // e4m3: [128] score constant of the row
   float* l_sh = rowc_sh + kTcRows;                                         // e4m3: [2][128] the sets' row sums
   float* scale_sh = l_sh + 2 * kTcRows;                                    // e4m3: [stage][4 c, 4 a, 4 1/v, 4 unused]
-  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2][4], buf[3] (+1 unused)
+  // full[], empty[], s[2], p[2], pv[2], sfree[2], m[2][4], buf[3] (+1 unused), s3[3] (+1 unused)
   uint64_t* bars = reinterpret_cast<uint64_t*>(ones_smem + kTcOnesBytes + kTcMBytes + kTcRowBytes + C::kScaleBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 20);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 24);
   int* cta_err = reinterpret_cast<int*>(tmem_slot + 1);
   int* rank_slot = cta_err + 1;
 
@@ -161,6 +163,12 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t bar_s = empty0 + 8 * kTcStages, bar_p = bar_s + 16, bar_pv = bar_p + 16;  // two of each
   const uint32_t bar_sfree = bar_pv + 16, bar_m = bar_sfree + 16;
   const uint32_t bar_buf = bar_m + 64;  // e4m3: S / P buffer k is free again (its P . V has completed)
+  // e4m3: S is ready in buffer k. One barrier per BUFFER, not per softmax set: the next S into a buffer needs
+  // the P . V of the one before, hence the softmax of the one before, so a barrier is never completed twice
+  // before its waiter has looked (with one per set, S(it + 2) -- which waits for no softmax warp here -- could
+  // complete the set's barrier a second time while the set had not yet waited for S(it), and a parity wait
+  // cannot tell phases two apart: a set was then left waiting for good)
+  const uint32_t bar_s3 = bar_buf + 32;
   if constexpr (!kFp8) {
     for (int i = tid; i < kTcOnesBytes / 4; i += kTcThreads)
       reinterpret_cast<uint32_t*>(ones_smem)[i] = 0x3F803F80u;  // 1.0 as bf16 pairs
@@ -179,7 +187,10 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
       for (int w = 0; w < 4; ++w) mbar_init(bar_m + 8 * (4 * k + w), 1);  // per warp: rows w*32.. of set k
     }
-    for (int k = 0; k < kFp8Bufs; ++k) mbar_init(bar_buf + 8 * k, 1);
+    for (int k = 0; k < kFp8Bufs; ++k) {
+      mbar_init(bar_buf + 8 * k, 1);
+      mbar_init(bar_s3 + 8 * k, 1);
+    }
     *cta_err = 0;
     fence_mbar_init();
     fence_proxy_async();
@@ -235,6 +246,12 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
   const uint32_t tmem_p = tmem_base + kTmemPBf16;  // bf16: P buffer k at tmem_p + 32 k (e4m3: P lies over its S)
 
   const int32_t* table = p.block_table + static_cast<int64_t>(b) * p.block_table_stride;
+  // e4m3, at most 64 query rows (e.g. 16 draft tokens x a group of 4): every row is held twice, in TMEM
+  // lanes r and r + 64, and the two copies share the softmax work of an iteration -- lane r takes its
+  // first 32 tokens, lane r + 64 the other 32, each as an online softmax of its own (own maximum, own row
+  // sum, own accumulator lane; the other half of its P is zero), merged at the end like split-KV partials.
+  // The softmax warps' chain per iteration, which bounds this kernel, is then half as long.
+  const bool half_rows = kFp8 && rows_total <= kTcRows / 2;
 
   // The roles, as closures.
   // ---- Q: row r -> (query token r / G, head r % G) goes to TMEM lane r as the A operand of S = Q . K^T
@@ -242,7 +259,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     // the two softmax warps that own the same 32 rows (w and w + 4) take half a row each
     if (warp < kTcSoftmaxWarps && (warp >> 2) < D / 64) {
       const int t = tid & (kTcRows - 1), half = warp >> 2;
-      const int r = rb * kTcRows + t;
+      const int r = half_rows ? (t & (kTcRows / 2 - 1)) : rb * kTcRows + t;
       const bool valid = r < rows_total;
       const int64_t qrow = (static_cast<int64_t>(b) * T + r / G) * p.num_q_heads + g * G + (r % G);
       const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow * D);
@@ -440,7 +457,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
           tc_mma_ts_if<false>(leader, d, u_tmem + kTmemQ<false> + 8 * ks, bd, idesc_s, ks > 0 ? 1u : 0u);
         }
       }
-      tc_commit_if(leader, bar_s + 8 * (it & 1));
+      tc_commit_if(leader, kFp8 ? bar_s3 + 8 * buf_i : bar_s + 8 * (it & 1));
       if (++stage_i == kTcStages) { stage_i = 0; stage_par ^= 1; }
       if (++buf_i == kFp8Bufs) { buf_i = 0; ++buf_round; }
     }
@@ -506,7 +523,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
   };
   auto softmax_role = [&]() {
-    // ================= softmax: TMEM lane t <-> query row t; set x takes iterations x, x+2, ... ==========
+    // ================= softmax on bf16 caches: TMEM lane t <-> query row t; set x takes iterations x, x+2, ...
     // Two warps per scheduler, one of each set: while one waits (for S, for the other set's row maximum,
     // for its tcgen05.ld/st) the other keeps the exp2 unit busy, which is what bounds this part.
     const int set = warp >> 2, t = tid & (kTcRows - 1);
@@ -520,12 +537,6 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     // the running maximum passes between the two warps that own the same 32 rows (same scheduler)
     const uint32_t my_m = bar_m + 8 * (4 * set + (warp & 3)), other_m = bar_m + 8 * (4 * (set ^ 1) + (warp & 3));
     float m_ref = -INFINITY;   // reference max the accumulated O and l are scaled by
-    // e4m3: this set's share of the row sum l (kept here, not in tensor memory) and the reference it is
-    // scaled by; the row's score constant (softmax scale, log2 e and the power of two Q was scaled by)
-    float l_set = 0.f, m_l = -INFINITY, rowc = 0.f;
-    if constexpr (kFp8) rowc = rowc_sh[t];
-    uint32_t sc_stage = set % kTcStages;  // ring stage of this set's next iteration
-    uint32_t my_buf = set;                 // e4m3: S / P buffer of this set's next iteration (it % 3)
     bool alive = true;
     auto fail = [&]() { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; };
     for (int it = set; it < n_iters; it += 2) {
@@ -535,17 +546,12 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       if (!ok) { fail(); break; }
       tc_fence_after();
       uint32_t sv[2][32];
-      const uint32_t sp_buf = tmem_s + 64 * (kFp8 ? my_buf : static_cast<uint32_t>(set)) + lane_base;
-      tmem_ld32(sp_buf, sv[0]);
-      tmem_ld32(sp_buf + 32, sv[1]);
+      tmem_ld32(tmem_s + 64 * set + lane_base, sv[0]);
+      tmem_ld32(tmem_s + 64 * set + lane_base + 32, sv[1]);
       tmem_wait_ld();
-      if constexpr (kFp8) {
-        my_buf = my_buf >= 1 ? my_buf - 1 : my_buf + 2;  // (it + 2) % 3
-      } else {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_tc(my_sfree);  // S(it) is in registers: S(it+2) may overwrite its buffer
-      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_tc(my_sfree);  // S(it) is in registers: S(it+2) may overwrite its buffer
       const int tok0 = (page0 + it * kTcPagesPerIter) * kPageSize;
       const int n_vis = min(lim, t1) - tok0;  // visible columns of this row in this iteration (may be <= 0)
       if (__any_sync(0xffffffffu, n_vis < kTcPagesPerIter * kPageSize)) {  // boundary tiles only
@@ -557,47 +563,14 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       // row maximum of the raw scores (the scale is positive), four independent chains
       float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      float mx;
-      // e4m3, per page j of the iteration: x = s cq[j] + aq[j] with cq = K scale x row constant and aq = log2
-      // of the V scale, i.e. the softmax runs on the scores plus log2(V scale): P then carries the V scale
-      // into P . V (V is multiplied as raw e4m3), and dividing the page's sum of P by the V scale (iq)
-      // gives its share of l.
-      float cq[4], aq[4], iq[4];
-      if constexpr (kFp8) {
-        // (written by the producer before the tiles' full barrier completed, which the S issue warp
-        // observed before the MMAs whose commit this warp has waited for)
-        const float4 c4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16);
-        const float4 a4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16 + 4);
-        const float4 i4 = *reinterpret_cast<const float4*>(scale_sh + sc_stage * 16 + 8);
-        // (kept above zero: a masked score, -inf, times 0 would be NaN)
-        cq[0] = fmaxf(c4.x * rowc, 1e-37f); cq[1] = fmaxf(c4.y * rowc, 1e-37f);
-        cq[2] = fmaxf(c4.z * rowc, 1e-37f); cq[3] = fmaxf(c4.w * rowc, 1e-37f);
-        aq[0] = a4.x; aq[1] = a4.y; aq[2] = a4.z; aq[3] = a4.w;
-        iq[0] = i4.x; iq[1] = i4.y; iq[2] = i4.z; iq[3] = i4.w;
-        sc_stage += 2;
-        if (sc_stage >= kTcStages) sc_stage -= kTcStages;
-        float mxb[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // two chains per page
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+      for (int h = 0; h < 2; ++h)
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const int q = h * 2 + (j >> 4);
-            mxs[q] = max3(mxs[q], __uint_as_float(sv[h][j]), __uint_as_float(sv[h][j + 1]));
-            mxb[q] = max3(mxb[q], __uint_as_float(sv[h][j + 2]), __uint_as_float(sv[h][j + 3]));
-          }
-        mx = fmaxf(fmaxf(fmaf(fmaxf(mxs[0], mxb[0]), cq[0], aq[0]), fmaf(fmaxf(mxs[1], mxb[1]), cq[1], aq[1])),
-                   fmaxf(fmaf(fmaxf(mxs[2], mxb[2]), cq[2], aq[2]), fmaf(fmaxf(mxs[3], mxb[3]), cq[3], aq[3])));
-      } else {
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-          for (int j = 0; j < 32; j += 2)
-            mxs[(j >> 1) & 3] = max3(mxs[(j >> 1) & 3], __uint_as_float(sv[h][j]), __uint_as_float(sv[h][j + 1]));
-        mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * scale_log2;
-      }
-      // bf16: the reference after iteration it-1 comes from the other set (one O for both). e4m3: each
-      // set runs an online softmax of its own over its iterations, with its own O.
-      if (!kFp8 && it > 0) {
+        for (int j = 0; j < 32; j += 2)
+          mxs[(j >> 1) & 3] = max3(mxs[(j >> 1) & 3], __uint_as_float(sv[h][j]), __uint_as_float(sv[h][j + 1]));
+      const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * scale_log2;
+      // the reference after iteration it-1 comes from the other set (one O for both)
+      if (it > 0) {
         ok = mbar_spin_bounded(other_m, ((it - 1) >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
@@ -605,28 +578,25 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       }
       // lazy rescaling: keep the old reference unless the max grew past the threshold
       float m_new = m_ref;
-      if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = kFp8 ? mx - kFp8RefBelowMax : fmaxf(m_ref, mx);
+      if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = fmaxf(m_ref, mx);
       const bool need = m_new != m_ref && m_ref != -INFINITY;
-      if constexpr (!kFp8) {
-        m_sh[(it & 1) * kTcRows + t] = m_new;
-        __syncwarp();
-        if (lane == 0) mbar_arrive_tc(my_m);  // (release: the other set reads m_sh after its wait)
-      }
-      if (it > (kFp8 ? 1 : 0) && __any_sync(0xffffffffu, need)) {
-        // O and l may only be touched once the last PV into them has completed: PV(it-1), or (e4m3)
-        // this set's PV(it-2). PV(it) is not issued before this warp arrives on bar_p below, and (bf16)
-        // the other set rescales only after PV(it)
+      m_sh[(it & 1) * kTcRows + t] = m_new;
+      __syncwarp();
+      if (lane == 0) mbar_arrive_tc(my_m);  // (release: the other set reads m_sh after its wait)
+      if (it > 0 && __any_sync(0xffffffffu, need)) {
+        // O and l may only be touched once the last PV into them, PV(it-1), has completed. PV(it) is not
+        // issued before this warp arrives on bar_p below, and the other set rescales only after PV(it)
         // (a parity wait tells neighbouring phases apart only: first this set's own PV(it-2), after which
         // the other set's barrier cannot be more than one phase behind)
         ok = it >= 2 ? mbar_spin_bounded(my_pv, (k - 1) & 1) : true;
-        if (!kFp8 && ok) ok = mbar_spin_bounded(bar_pv + 8 * (set ^ 1), ((it - 1) >> 1) & 1);
+        if (ok) ok = mbar_spin_bounded(bar_pv + 8 * (set ^ 1), ((it - 1) >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
         tc_fence_after();
         const float alpha = need ? ex2(m_ref - m_new) : 1.f;
-        const uint32_t my_o = tmem_o + (kFp8 ? D * set : 0) + lane_base;
+        const uint32_t my_o = tmem_o + lane_base;
 #pragma unroll
-        for (int cb = 0; cb < D / 32 + (kFp8 ? 0 : 1); ++cb) {  // O, then (bf16) the block of columns that holds l
+        for (int cb = 0; cb < D / 32 + 1; ++cb) {  // O, then the block of columns that holds l
           uint32_t ov[32];
           tmem_ld32(my_o + (cb < D / 32 ? 32 * cb : kTmemL - kTmemO<false>), ov);
           tmem_wait_ld();
@@ -639,41 +609,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       m_ref = m_new;
       const float ref = m_ref == -INFINITY ? 0.f : m_ref;
       uint32_t pw[32];
-      uint32_t pw_lo[kFp8 ? 16 : 1];  // e4m3: the low parts of P
-      if constexpr (kFp8) {
-        if (m_l != m_ref) {  // this set's row sum follows the reference (changed here or by the other set)
-          l_set *= ex2(m_l - m_ref);
-          m_l = m_ref;
-        }
-        // P = exp2(x - ref) as hi (e4m3) + mid (e4m3) + lo (e5m2), four tokens to a column: columns 0..15
-        // the high parts, 16..31 the middle parts, 32..47 the low parts (the A operands of the three
-        // P . V products)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint64_t c2 = f32x2(__float_as_uint(cq[q]), __float_as_uint(cq[q]));
-          const uint64_t nr2 = f32x2(__float_as_uint(aq[q] - ref), __float_as_uint(aq[q] - ref));
-          uint64_t sum2 = 0ull;
-#pragma unroll
-          for (int j = 8 * q; j < 8 * q + 8; j += 2) {  // two pairs = four tokens = one column
-            uint32_t hi[2], mid[2], lo[2];
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const uint64_t x2 = fma_f32x2(f32x2(sv[j >> 4][(2 * (j + e)) & 31], sv[j >> 4][(2 * (j + e) + 1) & 31]), c2, nr2);
-              float x0, x1;
-              f32x2_split(x2, x0, x1);
-              const float p0 = ex2(x0), p1 = ex2(x1);
-              sum2 = add_f32x2(sum2, f32x2(__float_as_uint(p0), __float_as_uint(p1)));
-              split_e4m3_e4m3_e5m2_x2(p0, p1, hi[e], mid[e], lo[e]);
-            }
-            pw[j >> 1] = hi[0] | (hi[1] << 16);
-            pw[16 + (j >> 1)] = mid[0] | (mid[1] << 16);
-            pw_lo[j >> 1] = lo[0] | (lo[1] << 16);
-          }
-          float s0, s1;
-          f32x2_split(sum2, s0, s1);
-          l_set = fmaf(s0 + s1, iq[q], l_set);
-        }
-      } else {
+      {
         // P = exp2(S * scale_log2 - ref) as bf16 pairs into TMEM lane t: the A operand of O += P . V
         // (one packed FMA per two elements; masked columns stay -inf -> 0)
         const uint64_t c2 = f32x2(__float_as_uint(scale_log2), __float_as_uint(scale_log2));
@@ -686,20 +622,12 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
           pw[j] = pack2<false>(ex2(x0), ex2(x1));
         }
       }
-      if (it >= 2) {
-        // bf16: PV(it-2) has finished reading the P buffer this iteration writes. (e4m3: P goes over its own
-        // S; the wait keeps this set's view of the barrier one phase behind at most, which the parity
-        // waits on it rely on)
+      if (it >= 2) {  // PV(it-2) has finished reading the P buffer this iteration writes
         ok = mbar_spin_bounded(my_pv, (k - 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { fail(); break; }
       }
-      if constexpr (kFp8) {
-        tmem_st32(sp_buf, pw);
-        tmem_st16(sp_buf + 32, pw_lo);
-      } else {
-        tmem_st32(tmem_p + 32 * set + lane_base, pw);
-      }
+      tmem_st32(tmem_p + 32 * set + lane_base, pw);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
@@ -708,19 +636,7 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
 
     // ---- finalise: the last iteration's reference (from the set that owned it) and the last PV
     bool ok = alive;
-    if constexpr (kFp8) {
-      // this set's last PV, then its (reference, row sum) for the merge of the two accumulators
-      const int last = n_iters - 1 - ((n_iters - 1 - set) & 1);  // its last iteration, if any
-      if (alive && last >= set) {
-        ok = mbar_wait_bounded(my_pv, (last >> 1) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
-        tc_fence_after();
-      }
-      if (m_l != m_ref) l_set *= ex2(m_l - m_ref);
-      m_sh[set * kTcRows + t] = m_ref;
-      l_sh[set * kTcRows + t] = l_set;
-    } else if (alive && n_iters > 0) {
+    if (alive && n_iters > 0) {
       const int last = n_iters - 1;
       if ((last & 1) != set) {
         ok = mbar_spin_bounded(bar_m + 8 * (4 * (last & 1) + (warp & 3)), (last >> 1) & 1);
@@ -741,23 +657,13 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     const int dev_err = max(err, *cta_err);
     if (dev_err && tid == 0) report(p.status, dev_err);
     const bool valid_row = r < rows_total;
-    bool have = alive && ok && n_iters > 0;  // warp-uniform
-    if constexpr (kFp8) have = have && *cta_err == 0;  // (the other set's view: its O is read below)
+    const bool have = alive && ok && n_iters > 0;  // warp-uniform
     float l = 0.f;
-    float w0 = 1.f, w1 = 0.f;  // e4m3: weights of the two sets' accumulators
     if (have) {
-      if constexpr (kFp8) {
-        const float m0 = m_sh[t], m1 = m_sh[kTcRows + t];
-        m_ref = fmaxf(m0, m1);
-        w0 = m0 == -INFINITY ? 0.f : ex2(m0 - m_ref);
-        w1 = m1 == -INFINITY ? 0.f : ex2(m1 - m_ref);
-        l = w0 * l_sh[t] + w1 * l_sh[kTcRows + t];
-      } else {
-        uint32_t lv[32];
-        tmem_ld32(tmem_base + kTmemL + lane_base, lv);
-        tmem_wait_ld();
-        l = __uint_as_float(lv[0]);
-      }
+      uint32_t lv[32];
+      tmem_ld32(tmem_base + kTmemL + lane_base, lv);
+      tmem_wait_ld();
+      l = __uint_as_float(lv[0]);
     }
     const bool live = !dev_err && have && l > 0.f;
     const float inv = live ? 1.f / l : 0.f;
@@ -770,17 +676,6 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       if (have) {
         tmem_ld32(tmem_o + lane_base + 32 * cb, ov);
         tmem_wait_ld();
-        if constexpr (kFp8) {  // O = w0 O[0] + w1 O[1] (the second exists from two iterations on)
-#pragma unroll
-          for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * w0);
-          if (n_iters > 1) {
-            uint32_t o1[32];
-            tmem_ld32(tmem_o + D + lane_base + 32 * cb, o1);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(fmaf(__uint_as_float(o1[j]), w1, __uint_as_float(ov[j])));
-          }
-        }
       } else {
 #pragma unroll
         for (int j = 0; j < 32; ++j) ov[j] = 0u;
@@ -809,6 +704,276 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     if (split && valid_row && set == 0)
       p.part_lse[qrow * p.max_chunks + p.chunk_slot0 + c] = live ? (m_ref + __log2f(l)) * kLn2 : -INFINITY;
   };
+  auto softmax_role_fp8 = [&](auto pages_tag) {
+    // ================= softmax on e4m3 caches. kNp = pages of an iteration a thread works on: 4 (its row
+    // sees all 64 tokens) or 2 (half rows: lanes below 64 take tokens 0..31, lanes from 64 tokens 32..63).
+    // Each set runs an online softmax of its own over its iterations, with its own O; nothing is
+    // exchanged per iteration.
+    constexpr int kNp = decltype(pages_tag)::value;
+    constexpr bool kHalf = kNp == 2;
+    constexpr int kNc = kNp * kPageSize;  // columns (tokens) per thread and iteration
+    const int set = warp >> 2, t = tid & (kTcRows - 1);
+    const int half = kHalf ? (t >> 6) : 0;  // warp-uniform
+    const int r = kHalf ? (t & (kTcRows / 2 - 1)) : rb * kTcRows + t;
+    const int i_tok = r / G;
+    const int lim = mp.causal ? min(L, L - T + i_tok + 1) : L;
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;  // this warp's TMEM lanes
+    const uint32_t my_p = bar_p + 8 * set, my_pv = bar_pv + 8 * set;
+    float m_ref = -INFINITY;   // reference the accumulated O is scaled by
+    // this thread's share of the row sum l (kept here, not in tensor memory) and the reference it is
+    // scaled by; the row's score constant (softmax scale, log2 e and the power of two Q was scaled by)
+    float l_set = 0.f, m_l = -INFINITY;
+    const float rowc = rowc_sh[t];
+    uint32_t sc_stage = set % kTcStages;  // ring stage of this set's next iteration
+    uint32_t my_buf = set;                 // S / P buffer of this set's next iteration (it % 3)
+    bool alive = true;
+    auto fail = [&]() { if (lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT); alive = false; };
+    for (int it = set; it < n_iters; it += 2) {
+      const int k = it >> 1;  // this set's k-th iteration: the phase index of its barriers
+      bool ok = mbar_spin_bounded(bar_s3 + 8 * my_buf, (static_cast<uint32_t>(it) / kFp8Bufs) & 1);  // S(it), buffer it % 3
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { fail(); break; }
+      tc_fence_after();
+      uint32_t sv[kNc];
+      const uint32_t sp_buf = tmem_s + 64 * my_buf + lane_base;
+      if constexpr (kHalf) {
+        tmem_ld32(sp_buf + 32 * half, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+      } else {
+        tmem_ld32(sp_buf, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+        tmem_ld32(sp_buf + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      }
+      tmem_wait_ld();
+      my_buf = my_buf >= 1 ? my_buf - 1 : my_buf + 2;  // (it + 2) % 3
+      const int tok0 = (page0 + it * kTcPagesPerIter) * kPageSize + kNc * half;  // first token of this thread's columns
+      const int n_vis = min(lim, t1) - tok0;  // visible ones among them (may be <= 0)
+      if (__any_sync(0xffffffffu, n_vis < kNc)) {  // boundary tiles only
+#pragma unroll
+        for (int j = 0; j < kNc; ++j) sv[j] = (j < n_vis) ? sv[j] : 0xff800000u;  // -inf
+      }
+      // per page j of the thread's columns: x = s cq[j] + aq[j] with cq = K scale x row constant and aq = log2 of
+      // the V scale, i.e. the softmax runs on the scores plus log2(V scale): P then carries the V scale
+      // into P . V (V is multiplied as raw e4m3), and dividing the page's sum of P by the V scale (iq)
+      // gives its share of l.
+      // (the constants were written by the producer before the tiles' full barrier completed, which the
+      // S issue warp observed before the MMAs whose commit this warp has waited for)
+      float cq[kNp], aq[kNp], iq[kNp];
+      {
+        const float* sc = scale_sh + sc_stage * 16 + kNp * half;
+#pragma unroll
+        for (int q = 0; q < kNp; ++q) {
+          cq[q] = fmaxf(sc[q] * rowc, 1e-37f);  // (kept above zero: a masked score, -inf, times 0 would be NaN)
+          aq[q] = sc[4 + q];
+          iq[q] = sc[8 + q];
+        }
+      }
+      sc_stage += 2;
+      if (sc_stage >= kTcStages) sc_stage -= kTcStages;
+      // row maximum of x over the thread's columns: per page the maximum of the raw scores (the factor is
+      // positive), two chains each
+      float mx = -INFINITY;
+#pragma unroll
+      for (int q = 0; q < kNp; ++q) {
+        float ma = -INFINITY, mb = -INFINITY;
+#pragma unroll
+        for (int j = 16 * q; j < 16 * q + 16; j += 4) {
+          ma = max3(ma, __uint_as_float(sv[j]), __uint_as_float(sv[j + 1]));
+          mb = max3(mb, __uint_as_float(sv[j + 2]), __uint_as_float(sv[j + 3]));
+        }
+        mx = fmaxf(mx, fmaf(fmaxf(ma, mb), cq[q], aq[q]));
+      }
+      // lazy rescaling: keep the old reference unless the max grew past the threshold; a new reference is
+      // set kFp8RefBelowMax under the maximum
+      float m_new = m_ref;
+      if (mx > m_ref + kRescaleThreshold || m_ref == -INFINITY) m_new = mx - kFp8RefBelowMax;
+      const bool need = m_new != m_ref && m_ref != -INFINITY;
+      if (it > 1 && __any_sync(0xffffffffu, need)) {
+        // O may only be touched once this set's last PV into it, PV(it-2), has completed; PV(it) is not
+        // issued before this warp arrives on bar_p below
+        ok = mbar_spin_bounded(my_pv, (k - 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { fail(); break; }
+        tc_fence_after();
+        const float alpha = need ? ex2(m_ref - m_new) : 1.f;
+        const uint32_t my_o = tmem_o + D * set + lane_base;
+#pragma unroll
+        for (int cb = 0; cb < D / 32; ++cb) {
+          uint32_t ov[32];
+          tmem_ld32(my_o + 32 * cb, ov);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
+          tmem_st32(my_o + 32 * cb, ov);
+        }
+        tmem_wait_st();
+      }
+      m_ref = m_new;
+      const float ref = m_ref == -INFINITY ? 0.f : m_ref;
+      if (m_l != m_ref) {  // the row sum follows the reference
+        l_set *= ex2(m_l - m_ref);
+        m_l = m_ref;
+      }
+      // P = exp2(x - ref) as hi (e4m3) + mid (e4m3) + lo (e5m2), four tokens to a column
+      uint32_t ph[4 * kNp], pm[4 * kNp], pl[4 * kNp];
+#pragma unroll
+      for (int q = 0; q < kNp; ++q) {
+        const uint64_t c2 = f32x2(__float_as_uint(cq[q]), __float_as_uint(cq[q]));
+        const uint64_t nr2 = f32x2(__float_as_uint(aq[q] - ref), __float_as_uint(aq[q] - ref));
+        uint64_t sum2 = 0ull;
+#pragma unroll
+        for (int j = 8 * q; j < 8 * q + 8; j += 2) {  // pairs j, j + 1 = four tokens = one column
+          uint16_t hi[2], mid[2], lo[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const uint64_t x2 = fma_f32x2(f32x2(sv[2 * (j + e)], sv[2 * (j + e) + 1]), c2, nr2);
+            float x0, x1;
+            f32x2_split(x2, x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            sum2 = add_f32x2(sum2, f32x2(__float_as_uint(p0), __float_as_uint(p1)));
+            split_e4m3_e4m3_e5m2_x2(p0, p1, hi[e], mid[e], lo[e]);
+          }
+          ph[j >> 1] = static_cast<uint32_t>(hi[0]) | (static_cast<uint32_t>(hi[1]) << 16);
+          pm[j >> 1] = static_cast<uint32_t>(mid[0]) | (static_cast<uint32_t>(mid[1]) << 16);
+          pl[j >> 1] = static_cast<uint32_t>(lo[0]) | (static_cast<uint32_t>(lo[1]) << 16);
+        }
+        float s0, s1;
+        f32x2_split(sum2, s0, s1);
+        l_set = fmaf(s0 + s1, iq[q], l_set);
+      }
+      if (it >= 2) {
+        // (P goes over its own S; this wait keeps the set's view of the barrier one phase behind at most,
+        // which the parity waits on it rely on)
+        ok = mbar_spin_bounded(my_pv, (k - 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { fail(); break; }
+      }
+      // columns 0..15 the high parts of the iteration's 64 tokens, 16..31 the middle parts, 32..47 the low
+      // parts (the A operands of the three P . V products); half rows: the other 32 tokens' columns are zero
+      if constexpr (kHalf) {
+        const uint32_t zeros[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        const uint32_t mine = sp_buf + 8 * half, other = sp_buf + 8 * (half ^ 1);  // (warp-uniform)
+        tmem_st8(mine, ph);       tmem_st8(other, zeros);
+        tmem_st8(mine + 16, pm);  tmem_st8(other + 16, zeros);
+        tmem_st8(mine + 32, pl);  tmem_st8(other + 32, zeros);
+      } else {
+        tmem_st16(sp_buf, ph);
+        tmem_st16(sp_buf + 16, pm);
+        tmem_st16(sp_buf + 32, pl);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_tc(my_p);
+    }
+
+    // ---- finalise: this set's last PV, then the merge of the accumulators that hold parts of a row: the
+    // two sets' (and, with half rows, those of lanes r and r + 64)
+    bool ok = alive;
+    {
+      const int last = n_iters - 1 - ((n_iters - 1 - set) & 1);  // this set's last iteration, if any
+      if (alive && last >= set) {
+        ok = mbar_wait_bounded(my_pv, (last >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok && lane == 0) atomicMax(cta_err, PDA_DEV_TIMEOUT);
+        tc_fence_after();
+      }
+      if (m_l != m_ref) l_set *= ex2(m_l - m_ref);
+      m_sh[set * kTcRows + t] = m_ref;
+      l_sh[set * kTcRows + t] = l_set;
+    }
+    // every softmax warp reaches this point together with its error view settled; all P . V have completed
+    asm volatile("bar.sync 2, %0;" ::"n"(kTcSoftmaxWarps * 32) : "memory");
+    const int dev_err = max(err, *cta_err);
+    if (dev_err && tid == 0) report(p.status, dev_err);
+    const bool valid_row = r < rows_total;
+    const bool have = alive && ok && n_iters > 0 && *cta_err == 0;  // warp-uniform (and CTA-uniform: cta_err is settled)
+    float l = 0.f, w0 = 0.f, w1 = 0.f;  // weights of this lane's two accumulators (one per set)
+    if (have) {
+      const float m0 = m_sh[t], m1 = m_sh[kTcRows + t];
+      float M = fmaxf(m0, m1);
+      const int tp = t ^ (kTcRows / 2);  // half rows: the lane that holds the row's other half
+      if constexpr (kHalf) M = fmaxf(M, fmaxf(m_sh[tp], m_sh[kTcRows + tp]));
+      auto wgt = [&](float m) { return m == -INFINITY ? 0.f : ex2(m - M); };
+      w0 = wgt(m0);
+      w1 = wgt(m1);
+      l = w0 * l_sh[t] + w1 * l_sh[kTcRows + t];
+      if constexpr (kHalf) l += wgt(m_sh[tp]) * l_sh[tp] + wgt(m_sh[kTcRows + tp]) * l_sh[kTcRows + tp];
+      m_ref = M;
+    }
+    const bool live = !dev_err && have && l > 0.f;
+    const float inv = live ? 1.f / l : 0.f;
+    const int64_t qrow = (static_cast<int64_t>(b) * T + i_tok) * p.num_q_heads + g * G + (r % G);
+    constexpr float kLn2 = 0.6931471805599453f;
+    // set x handles columns [D/2 x, D/2 (x + 1)) of the row, 32 at a time: this lane's accumulators, weighted
+    uint32_t ov[D / 64][32];
+#pragma unroll
+    for (int cc = 0; cc < D / 64; ++cc) {
+      const int cb = (D / 64) * set + cc;
+      if (have) {
+        tmem_ld32(tmem_o + lane_base + 32 * cb, ov[cc]);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ov[cc][j] = __float_as_uint(__uint_as_float(ov[cc][j]) * w0);
+        if (n_iters > 1) {  // (the second set's accumulator exists from two iterations on)
+          uint32_t o1[32];
+          tmem_ld32(tmem_o + D + lane_base + 32 * cb, o1);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            ov[cc][j] = __float_as_uint(fmaf(__uint_as_float(o1[j]), w1, __uint_as_float(ov[cc][j])));
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ov[cc][j] = 0u;
+      }
+    }
+    if constexpr (kHalf) {
+      // lanes from 64 hand their part to the lane that stores the row, through the idle ring
+      // ([column][row]: a warp's lanes write consecutive words)
+      float* xch = reinterpret_cast<float*>(smem);
+      if (half == 1) {
+#pragma unroll
+        for (int cc = 0; cc < D / 64; ++cc)
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            xch[(((D / 64) * set + cc) * 32 + j) * (kTcRows / 2) + (t & (kTcRows / 2 - 1))] = __uint_as_float(ov[cc][j]);
+      }
+      asm volatile("bar.sync 2, %0;" ::"n"(kTcSoftmaxWarps * 32) : "memory");
+      if (half == 0) {
+#pragma unroll
+        for (int cc = 0; cc < D / 64; ++cc)
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            ov[cc][j] = __float_as_uint(__uint_as_float(ov[cc][j]) +
+                                        xch[(((D / 64) * set + cc) * 32 + j) * (kTcRows / 2) + t]);
+      }
+    }
+    if (valid_row && half == 0) {
+#pragma unroll
+      for (int cc = 0; cc < D / 64; ++cc) {
+        const int cb = (D / 64) * set + cc;
+        if (split) {
+          float4* dst = reinterpret_cast<float4*>(p.part_o + (qrow * p.max_chunks + p.chunk_slot0 + c) * D + 32 * cb);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            dst[j] = make_float4(__uint_as_float(ov[cc][4 * j]) * inv, __uint_as_float(ov[cc][4 * j + 1]) * inv,
+                                 __uint_as_float(ov[cc][4 * j + 2]) * inv, __uint_as_float(ov[cc][4 * j + 3]) * inv);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(p.out + qrow * D + 32 * cb);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              w[e] = pack2<false>(__uint_as_float(ov[cc][8 * j + 2 * e]) * inv,
+                                  __uint_as_float(ov[cc][8 * j + 2 * e + 1]) * inv);
+            dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      if (split && set == 0)
+        p.part_lse[qrow * p.max_chunks + p.chunk_slot0 + c] = live ? (m_ref + __log2f(l)) * kLn2 : -INFINITY;
+    }
+  };
   if constexpr (!kFp8) {
     load_q();
     if (warp == kTcProducerWarp) producer_role(); else wait_q();
@@ -822,7 +987,8 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
       reg_alloc_inc<kTcRegsSoftmax>();
       load_q();
       wait_q();
-      softmax_role();
+      if (half_rows) softmax_role_fp8(std::integral_constant<int, 2>{});
+      else softmax_role_fp8(std::integral_constant<int, 4>{});
     } else {
       reg_alloc_dec<kTcRegsControl>();
       if (warp == kTcProducerWarp) {

@@ -82,20 +82,16 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
 // is left (at most three) fits e5m2: the three parts add up to f16(x) exactly as long as no part falls
 // below its format's range, i.e. for x >= 2^-6. Below that e4m3's subnormal step of 2^-9 takes bits from
 // hi and mid and the sum is within 2^-7 x, never worse than 2^-17.
-__device__ __forceinline__ void split_e4m3_e4m3_e5m2_x2(float x0, float x1, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
+__device__ __forceinline__ void split_e4m3_e4m3_e5m2_x2(float x0, float x1, uint16_t& hi, uint16_t& mid, uint16_t& lo) {
   uint32_t xh, back;
-  uint16_t h, m, l;
   asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(xh) : "f"(x1), "f"(x0));
-  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(h) : "r"(xh));
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(h));
+  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(hi) : "r"(xh));
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(hi));
   asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(xh) : "r"(xh), "r"(back));
-  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(m) : "r"(xh));
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(m));
+  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(mid) : "r"(xh));
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(mid));
   asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(xh) : "r"(xh), "r"(back));
-  asm("cvt.rn.satfinite.e5m2x2.f16x2 %0, %1;" : "=h"(l) : "r"(xh));
-  hi = h;
-  mid = m;
-  lo = l;
+  asm("cvt.rn.satfinite.e5m2x2.f16x2 %0, %1;" : "=h"(lo) : "r"(xh));
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -118,6 +114,12 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
         "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
       : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
