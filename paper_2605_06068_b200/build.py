@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libpda.so")
-SOURCES = ["api.cu", "kv_append.cu", "reduce.cu", "attention_generic.cu", "attention_tma.cu", "attention_persist.cu", "attention_mq.cu", "attention_mq_tc.cu", "attention_mq_tcp.cu",
+SOURCES = ["api.cu", "kv_append.cu", "reduce.cu", "attention_generic.cu", "attention_tma.cu", "attention_persist.cu", "attention_mq.cu", "attention_mq_tc.cu", "attention_mq_tcp.cu", "attention_mq_tc8p.cu",
            "static_scratch.cu", "debug.cu"]
 
 NVCC_FLAGS = [

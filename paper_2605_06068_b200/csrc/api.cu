@@ -325,6 +325,8 @@ int paged_verify_attention(const void* q, const void* k_cache, const void* v_cac
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (!(flags & (PDA_FLAG_MQ_MMA_SYNC | PDA_FLAG_MQ_ONE_UNIT)) && pda::attention_mq_tcp_supports(mp)) {
     if (cudaError_t e = pda::launch_attention_mq_tcp(mp, s)) return static_cast<int>(e);
+  } else if (!(flags & (PDA_FLAG_MQ_MMA_SYNC | PDA_FLAG_MQ_ONE_UNIT)) && pda::attention_mq_tc8p_supports(mp)) {
+    if (cudaError_t e = pda::launch_attention_mq_tc8p(mp, s)) return static_cast<int>(e);
   } else if (!(flags & PDA_FLAG_MQ_MMA_SYNC) && pda::attention_mq_tc_supports(mp)) {
     if (cudaError_t e = pda::launch_attention_mq_tc(mp, s)) return static_cast<int>(e);
   } else {

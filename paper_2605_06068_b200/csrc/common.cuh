@@ -121,6 +121,9 @@ bool attention_mq_tc_supports(const MqParams& mp);
 cudaError_t launch_attention_mq_tc(const MqParams& mp, cudaStream_t stream);
 bool attention_mq_tcp_supports(const MqParams& mp);
 cudaError_t launch_attention_mq_tcp(const MqParams& mp, cudaStream_t stream);
+// persistent tcgen05 + TMEM version for e4m3 KV (head_dim 128, unsplit)
+bool attention_mq_tc8p_supports(const MqParams& mp);
+cudaError_t launch_attention_mq_tc8p(const MqParams& mp, cudaStream_t stream);
 cudaError_t launch_attention_mq(const MqParams& mp, cudaStream_t stream);
 cudaError_t launch_kv_append_tokens(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                     const CacheGeom& g, const int32_t* block_table, int32_t bt_stride,
