@@ -403,13 +403,15 @@ attention_mq_tc_kernel(const __grid_constant__ CUtensorMap k_map,
     uint32_t buf_i = 0, buf_round = 0;    // e4m3: it % 3 and it / 3
     for (int it = 0; it < u_iters; ++it) {
       if constexpr (kFp8) {
+        // (the stage first: it has landed long ago as a rule, while the buffer is what S waits for)
+        ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);  // the block has landed
         // S(it) overwrites the buffer of S(it-3) and P(it-3): P(it-3) . V has completed
-        if (it >= kFp8Bufs) ok = mbar_wait_bounded(bar_buf + 8 * buf_i, (buf_round - 1) & 1);
+        if (ok && it >= kFp8Bufs) ok = mbar_wait_bounded(bar_buf + 8 * buf_i, (buf_round - 1) & 1);
       } else {
         // S(it) overwrites the buffer of S(it-2): the softmax warps have loaded that into registers
         if (it >= 2) ok = mbar_wait_bounded(bar_sfree + 8 * (it & 1), ((it - 2) >> 1) & 1);
+        if (ok) ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);  // the block has landed
       }
-      if (ok) ok = mbar_wait_bounded(full0 + 8 * stage_i, stage_par);  // the block has landed
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const uint32_t stage = ring + stage_i * C::kOperandBytes;

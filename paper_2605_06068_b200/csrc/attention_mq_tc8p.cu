@@ -33,8 +33,10 @@ constexpr int kETileBytes = kPageSize * kED;          // one K or V page tile: 2
 constexpr int kEKBytes = kEPagesPerIter * kETileBytes;  // K of 4 pages: [64 tokens][128 B]
 constexpr int kEStageBytes = 2 * kEKBytes;            // K block, then 4 V page tiles: 16 KB
 constexpr int kEStages = 11;
-constexpr int kEQxBytes = 32768;                      // staged Q: [row][128 B high parts | 128 B low parts]; half rows:
-                                                      // 64 rows of it, then 16 KB for the exchange between lanes r + 64 and r
+constexpr int kEQPitch = 272;                         // staged Q row: 128 B high parts | 128 B low parts | 16 B pad, so that
+                                                      // a warp's 16-byte accesses to 32 rows spread over all banks
+constexpr int kEQxBytes = kERows * kEQPitch;          // the stage; half rows: 64 rows of it, then an area of the same size
+                                                      // for the exchange between lanes r + 64 and r and for the output rows
 constexpr int kEMaxBatch = 1024;                      // lengths and order of the sequences in shared memory
 constexpr int kEBars = 2 * kEStages + 3 + 2 + 2 + 3 + 3;  // full, empty, s3, p, pv, buf, q / qfull / qfree
 constexpr int kESmemBytes = kEStages * kEStageBytes + kEQxBytes + 2 * kERows * 4 /* m */ + 2 * kERows * 4 /* l */ +
@@ -180,8 +182,8 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
         const int up = (ex == 0 || ex == 255) ? 0 : min(max(134 - ex, -100), 100);  // it times 2^up is in [128, 256)
         const float mul = __uint_as_float(static_cast<uint32_t>(127 + up) << 23);
         rowc_st[t] = p.scale * 1.4426950408889634f * __uint_as_float(static_cast<uint32_t>(127 - up) << 23);
-        uint2* dst_hi = reinterpret_cast<uint2*>(qx + t * 256);
-        uint2* dst_lo = reinterpret_cast<uint2*>(qx + t * 256 + 128);
+        uint2* dst_hi = reinterpret_cast<uint2*>(qx + t * kEQPitch);
+        uint2* dst_lo = reinterpret_cast<uint2*>(qx + t * kEQPitch + 128);
 #pragma unroll 2
         for (int ch = 0; ch < D / 8; ++ch) {  // (the second pass over the row comes from L1 / L2)
           const uint4 v = valid ? __ldg(src + ch) : make_uint4(0u, 0u, 0u, 0u);
@@ -283,8 +285,9 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
       for (int it = 0; it < u.n_iters; ++it, ++gi) {
         const uint32_t buf = gi % kEBufs, s = gi % kEStages;
         // S(gi) overwrites the buffer of S(gi-3) and P(gi-3): P(gi-3) . V has completed
-        if (gi >= kEBufs) ok = mbar_wait_bounded(bar_buf + 8 * buf, ((gi / kEBufs) - 1) & 1);
-        if (ok) ok = mbar_wait_bounded(full0 + 8 * s, (gi / kEStages) & 1);  // the block has landed
+        // (the stage first: it has landed long ago as a rule, while the buffer is what S waits for)
+        ok = mbar_wait_bounded(full0 + 8 * s, (gi / kEStages) & 1);  // the block has landed
+        if (ok && gi >= kEBufs) ok = mbar_wait_bounded(bar_buf + 8 * buf, ((gi / kEBufs) - 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         const uint32_t stage = ring + s * kEStageBytes;
@@ -386,8 +389,8 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
       float rowc = 0.f;
       if (alive) {
         uint32_t qh[16], ql[16];
-        const uint4* sh = reinterpret_cast<const uint4*>(qx + qr * 256 + 64 * set);
-        const uint4* sl = reinterpret_cast<const uint4*>(qx + qr * 256 + 128 + 64 * set);
+        const uint4* sh = reinterpret_cast<const uint4*>(qx + qr * kEQPitch + 64 * set);
+        const uint4* sl = reinterpret_cast<const uint4*>(qx + qr * kEQPitch + 128 + 64 * set);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint4 a = sh[i], b4 = sl[i];
@@ -616,7 +619,7 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
       if constexpr (kHalf) {
         // lanes from 64 hand their part to the lane that stores the row, 32 columns per set at a time, through
         // the second half of the Q staging area ([set][column][row]: a warp's lanes write consecutive words)
-        float* xch = reinterpret_cast<float*>(qx + kEQxBytes / 2);
+        float* xch = reinterpret_cast<float*>(qx + kEQxBytes / 2);  // (16 KB of that area)
 #pragma unroll
         for (int cc = 0; cc < D / 64; ++cc) {
           if (half == 1) {
@@ -636,7 +639,38 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
       } else {
         asm volatile("bar.sync 2, %0;" ::"n"(kESoftmaxWarps * 32) : "memory");  // the unit's closing barrier
       }
-      if (valid_row && half == 0) {
+      if constexpr (kHalf) {
+        // The rows leave through shared memory (the exchange area is free again): a thread holds 64 columns
+        // of one row, so stored directly a warp's instruction would touch 32 rows; from shared memory every
+        // 16 lanes write one row's 256 bytes.
+        uint8_t* ostage = qx + kEQxBytes / 2;
+        if (half == 0) {
+          uint4* dst = reinterpret_cast<uint4*>(ostage + qr * kEQPitch + 128 * set);
+#pragma unroll
+          for (int cc = 0; cc < D / 64; ++cc)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                w[e] = pack2<false>(__uint_as_float(ov[cc][8 * j + 2 * e]) * inv,
+                                    __uint_as_float(ov[cc][8 * j + 2 * e + 1]) * inv);
+              dst[4 * cc + j] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        asm volatile("bar.sync 2, %0;" ::"n"(kESoftmaxWarps * 32) : "memory");
+#pragma unroll
+        for (int k = 0; k < (kERows / 2) * 16 / (kESoftmaxWarps * 32); ++k) {
+          const int chunk = tid + k * kESoftmaxWarps * 32;  // 16-byte piece of the 64 x 256 bytes
+          const int row = chunk >> 4, piece = chunk & 15;
+          const int rr = u.rb * kERows + row;
+          if (rr < rows_total) {
+            const int64_t orow = (static_cast<int64_t>(u.b) * T + rr / G) * p.num_q_heads + u.g * G + (rr % G);
+            *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out + orow * D) + 16 * piece) =
+                *reinterpret_cast<const uint4*>(ostage + row * kEQPitch + 16 * piece);
+          }
+        }
+      } else if (valid_row) {
         const int64_t qrow = (static_cast<int64_t>(u.b) * T + i_tok) * p.num_q_heads + u.g * G + (r % G);
 #pragma unroll
         for (int cc = 0; cc < D / 64; ++cc) {
