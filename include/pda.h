@@ -424,7 +424,8 @@ int pda_debug_e4m3_decode(float* out256, pda_stream_t stream);
  * unit's output and returns. This call launches one warp that initialises such a
  * barrier, never arrives at it, and runs the same two wait helpers (the suspended
  * try_wait form of the TMA rings, the spinning test_wait form of the tensor-core
- * hand-offs) with `polls` as their limit instead of the built-in 2^20 and 2^24.
+ * hand-offs) with `polls` as their limit instead of the built-in 2^18 (4.0 us per
+ * poll: 1.05 s) and 2^24 (21.9 ns per poll: 0.37 s).
  * Nothing faults and nothing waits without a limit; the context stays usable.
  *   polls   1 .. 2^20
  *   status  device int32: receives atomicMax(PDA_DEV_TIMEOUT)

@@ -61,7 +61,7 @@ __device__ __forceinline__ void publish_unit(volatile int* ring_sh, int k, int p
 __device__ __forceinline__ int unit_entry(volatile int* ring_sh, int k, int lane) {  // a whole warp; -2: timed out
   int pos = -2;
   if (lane == 0) {
-    for (uint32_t i = 0; i < (1u << 24); ++i) {
+    for (uint32_t i = 0; i < (1u << 23); ++i) {  // (64 ns naps: gives up after about a second)
       if (ring_sh[2 * (k % kPClaimRing)] == k + 1) {
         __threadfence_block();
         pos = ring_sh[2 * (k % kPClaimRing) + 1];

@@ -11,7 +11,7 @@ constexpr int kUmmaRows = 128;  // UMMA M: query rows per CTA, one TMEM lane eac
 
 // Spinning bounded wait (no suspension): the waits on the MMA/softmax hand-off are short and on the
 // critical path, where the wake-up latency of a suspended try_wait shows. A poll is a test_wait and its
-// loop overhead, some tens of clocks: 2^24 of them give up after a few tenths of a second.
+// loop overhead, 21.9 ns measured (pda_debug_wait_timeout): 2^24 of them give up after 0.37 s.
 constexpr uint32_t kTestSpinLimit = 1u << 24;
 __device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kTestSpinLimit) {
   for (uint32_t i = 0; i < limit; ++i)
