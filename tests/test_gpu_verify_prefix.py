@@ -343,3 +343,65 @@ def test_verify_persistent_kernel_in_a_cuda_graph(oracle):
         torch.cuda.synchronize()
         assert torch.equal(out.view(torch.int16), eager.view(torch.int16))
     assert int(dw.status.item()) == 0
+
+
+@pytest.mark.parametrize("T", [8, 40])
+def test_verify_fp8_persistent_kernel_edge_cases(oracle, T):
+    """The persistent e4m3 kernel (the default for unsplit calls on e4m3 caches): more units than SMs, so
+    that every CTA walks through several; sequences that are empty, shorter than the block, and one
+    token on either side of a page and of an iteration; 32 query rows per kv head (rows held twice, T = 8)
+    and 160 (two row blocks, T = 40). Then a page id outside the pool and a length beyond the table: the
+    status word reports them, those sequences' rows are zero and every other row is right. Last, the
+    launch captured in a CUDA graph and replayed."""
+    lens = [0, 3, 16, 17, 63, 64, 65, 700, 1, 129, 256, 300] + [30 + 11 * i for i in range(28)]   # 40 x 8 units
+    w = W.make_workload("fp8_units", lens, 32, 8, 128, kv_dtype="e4m3", seed=171)
+    q, _, _ = verify_inputs(w, T, 172)
+    ref, _ = oracle.paged_verify_attention(q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.scale,
+                                           w.k_scale, w.v_scale)
+    dw = DeviceWorkload(w)
+    dq = bf16_tensor(q)
+    out = pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, float(w.scale),
+                                     k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status)
+    got = bf16_to_f64(out)
+    assert_close(got, ref, "e4m3", what=f"persistent e4m3 verify T={T}")
+    assert (got[0] == 0).all() and int(dw.status.item()) == 0        # the empty sequence's rows are zero
+    one_unit = pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, float(w.scale),
+                                          k_scale=dw.k_scale, v_scale=dw.v_scale, flags=pda.PDA_FLAG_MQ_ONE_UNIT)
+    # the same arithmetic unit by unit (which softmax set takes which iteration differs, so not bit for bit)
+    assert_close(bf16_to_f64(one_unit), ref, "e4m3", what=f"one-unit e4m3 verify T={T}")
+    assert np.abs(bf16_to_f64(one_unit) - got).max() <= 4e-3
+    # bad inputs
+    bt = dw.block_table.clone()
+    bt[7, 5] = w.num_pages + 3
+    bt[10, 0] = -1
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bad = bf16_to_f64(pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, bt, dw.seq_lens, float(w.scale),
+                                                 k_scale=dw.k_scale, v_scale=dw.v_scale, status=st))
+    assert int(st.item()) == 1      # PDA_DEV_BAD_PAGE
+    good = [b for b in range(len(lens)) if b not in (7, 10)]
+    assert_close(bad[good], ref[good], "e4m3", what="rows beside a bad table row")
+    assert (bad[[7, 10]] == 0).all()
+    sl = dw.seq_lens.clone()
+    sl[11] = bt.shape[1] * 16 + 9
+    st.zero_()
+    bad = bf16_to_f64(pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, sl, float(w.scale),
+                                                 k_scale=dw.k_scale, v_scale=dw.v_scale, status=st))
+    assert int(st.item()) == 2      # PDA_DEV_BAD_SEQ_LEN
+    good = [b for b in range(len(lens)) if b != 11]
+    assert_close(bad[good], ref[good], "e4m3", what="rows beside a bad length")
+    assert (bad[11] == 0).all()
+    # captured and replayed
+    res = torch.empty_like(dq)
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            pda.paged_verify_attention(dq, dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, float(w.scale),
+                                       out=res, k_scale=dw.k_scale, v_scale=dw.v_scale, status=dw.status, stream=s)
+    for _ in range(3):
+        res.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(res.view(torch.int16), out.view(torch.int16))
+    assert int(dw.status.item()) == 0
