@@ -79,7 +79,7 @@ extern "C" {
 #define PDA_FLAG_MQ_MMA_SYNC 2u   /* multi-query calls (verify, shared prefix): use the mma.sync
                                      kernel even where the tcgen05 + TMEM kernel applies */
 #define PDA_FLAG_MQ_ONE_UNIT 4u   /* paged_verify_attention: one CTA per (sequence, kv head, row block) even
-                                     where the persistent tcgen05 kernel applies (unsplit, bf16, head_dim 128) */
+                                     where a persistent tcgen05 kernel applies (unsplit, head_dim 128) */
 
 typedef void* pda_stream_t; /* cudaStream_t */
 
@@ -230,10 +230,10 @@ int kv_append_tokens_fp8(const void* k_new, const void* v_new, void* k_cache, vo
  * group size), so each page is fetched once per block, not once per token.
  * bf16 KV with head_dim 128 or 64 and e4m3 KV with head_dim 128 run on tcgen05
  * tensor-core tiles with the accumulators in tensor memory (128 query rows per CTA);
- * PDA_FLAG_MQ_MMA_SYNC selects the mma.sync kernel instead. Unsplit calls on bf16
- * caches with head_dim 128 and up to 1024 sequences run as one persistent CTA per SM
- * that walks through the (sequence, kv head, row block) units, longest sequences
- * first (PDA_FLAG_MQ_ONE_UNIT: one CTA per unit). That kernel shares out its last
+ * PDA_FLAG_MQ_MMA_SYNC selects the mma.sync kernel instead. Unsplit calls with
+ * head_dim 128 and up to 1024 sequences run as one persistent CTA per SM that walks
+ * through the (sequence, kv head, row block) units, longest sequences first
+ * (PDA_FLAG_MQ_ONE_UNIT: one CTA per unit). The bf16 one of these kernels shares out its last
  * units through a counter in device memory which the library owns (a pool of 64,
  * taken in turn by the launches and left at zero by each): up to 64 such launches
  * may be in flight at once on a device; a launch captured in a CUDA graph keeps its
