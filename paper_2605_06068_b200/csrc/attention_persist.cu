@@ -123,13 +123,14 @@ attention_persist_kernel(const __grid_constant__ CUtensorMap k_map,
     }
   };
   const uint32_t leader = elect_one();
+  const uint64_t pol = l2_policy_evict_first();  // the tiles are read once: first out of the L2
   auto issue = [&](uint32_t ordinal, int g, int page_raw) {  // whole warp, converged; the elected lane issues
     const int s = ordinal % kStages;
     const uint32_t bar = bar0 + 8 * s;
     const uint32_t dst = ring + s * C::kStageBytes;
     mbar_expect_tx_if(leader, bar, C::kStageBytes);
-    tma_load_5d_if(leader, dst, &k_map, bar, 0, g, max(page_raw, 0));
-    tma_load_5d_if(leader, dst + C::kTileBytes, &v_map, bar, 0, g, max(page_raw, 0));
+    tma_load_5d_hint_if(leader, dst, &k_map, bar, 0, g, max(page_raw, 0), pol);
+    tma_load_5d_hint_if(leader, dst + C::kTileBytes, &v_map, bar, 0, g, max(page_raw, 0), pol);
   };
 
   const float scale_log2 = p.scale * 1.4426950408889634f;

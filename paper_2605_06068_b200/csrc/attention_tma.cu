@@ -152,14 +152,15 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
   load_block(1, pgB, ksB, vsB);
 
   const uint32_t leader = elect_one();
+  const uint64_t pol = l2_policy_evict_first();
   auto issue = [&](int kk, int page_raw) {  // whole warp, converged; the elected lane issues
     const int page = max(page_raw, 0);
     const int s = kk % kStages;
     const uint32_t bar = bar0 + 8 * s;
     const uint32_t dst = ring + s * C::kStageBytes;
     mbar_expect_tx_if(leader, bar, C::kStageBytes);
-    tma_load_5d_if(leader, dst, &k_map, bar, 0, g, page);
-    tma_load_5d_if(leader, dst + C::kTileBytes, &v_map, bar, 0, g, page);
+    tma_load_5d_hint_if(leader, dst, &k_map, bar, 0, g, page, pol);
+    tma_load_5d_hint_if(leader, dst + C::kTileBytes, &v_map, bar, 0, g, page, pol);
   };
 
   // prologue: fill the ring

@@ -81,6 +81,20 @@ __device__ __forceinline__ void tma_load_5d_if(uint32_t leader, uint32_t dst, co
       " [%0], [%1, {0, 0, %3, %4, %5}], [%2];\n\t}"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c2), "r"(c3), "r"(c4), "r"(leader) : "memory");
 }
+// The same with an L2 cache policy (from createpolicy): for tiles that are read once.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_5d_hint_if(uint32_t leader, uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                    int c2, int c3, int c4, uint64_t policy) {
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %6, 0;\n\t"
+      "@pe cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {0, 0, %3, %4, %5}], [%2], %7;\n\t}"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c2), "r"(c3), "r"(c4), "r"(leader), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx_if(uint32_t leader, uint32_t bar, uint32_t bytes) {
   asm volatile(
       "{\n\t.reg .pred pe;\n\tsetp.ne.b32 pe, %2, 0;\n\t"
