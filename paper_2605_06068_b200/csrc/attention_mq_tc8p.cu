@@ -209,6 +209,8 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
   // ---- TMA producer: runs through all units of the CTA, held back only by the ring
   auto producer_role = [&]() {
     const uint32_t leader = elect_one();
+    const uint64_t pol = l2_policy_evict_first();  // a sequence's own tiles are read once; a shared prefix stays
+                                                   // in the L2 all the same (measured)
     EUnit u;
     uint32_t gi = 0;  // iterations so far, over all units
     bool bad = false, alive = true;
@@ -255,8 +257,8 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
           const int page_raw = __shfl_sync(0xffffffffu, pg, (it & 7) * kEPagesPerIter + j);
           bad |= page_raw < 0;
           const int page = max(page_raw, 0);
-          tma_load_5d_if(leader, stage + j * kETileBytes, &k_map, bar, 0, g, page);
-          tma_load_5d_if(leader, stage + kEKBytes + j * kETileBytes, &v_map, bar, 0, g, page);
+          tma_load_5d_hint_if(leader, stage + j * kETileBytes, &k_map, bar, 0, g, page, pol);
+          tma_load_5d_hint_if(leader, stage + kEKBytes + j * kETileBytes, &v_map, bar, 0, g, page, pol);
         };
         if (n_here == kEPagesPerIter) {
 #pragma unroll

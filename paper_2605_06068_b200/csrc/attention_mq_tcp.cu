@@ -182,6 +182,7 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
   if (warp == kPProducerWarp) {
     // ================= TMA producer: runs through the units' tiles, up to kPStages iterations ahead ====
     const uint32_t leader = elect_one();
+    const uint64_t pol = l2_policy_evict_first();  // the tiles are read once: first out of the L2
     bool bad = false, dead = false;
     uint32_t gi = 0;
     // (a quarter of the rounds, at most kPClaimedRounds: with only three or four units a CTA the deal is as
@@ -257,8 +258,8 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
           const int page = max(page_raw, 0);
 #pragma unroll
           for (int ln = 0; ln < kPLines; ++ln)
-            tma_load_5d_if(leader, stage + ln * (kPKBytes / kPLines) + j * (kPageSize * 128), &k_map, bar, ln, u.g, page);
-          tma_load_5d_if(leader, stage + kPKBytes + j * kPTileBytes, &v_map, bar, 0, u.g, page);
+            tma_load_5d_hint_if(leader, stage + ln * (kPKBytes / kPLines) + j * (kPageSize * 128), &k_map, bar, ln, u.g, page, pol);
+          tma_load_5d_hint_if(leader, stage + kPKBytes + j * kPTileBytes, &v_map, bar, 0, u.g, page, pol);
         };
         if (n_here == kPPagesPerIter) {
 #pragma unroll
