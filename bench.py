@@ -52,7 +52,7 @@ DEFAULT_ALSO = ["longctx", "chat70b", "prefix_fp8"]
 # from the ncu captures summarised under profiles/ (None: not captured). Captures taken on a batch cut
 # to about 1 GB are scaled to the full batch by the KV bytes (traffic grows with them).
 NCU_TRAFFIC_BYTES = {
-    "llama8b": 621_190_000,       # profiles/attention_tma_llama8b_ncu.md
+    "llama8b": 620_500_000,       # profiles/attention_tma_llama8b_ncu.md
     "longctx": 2_707_000_000,     # profiles/attention_tma_split_fused_longctx_ncu.md (2 of 8 sequences captured, x 4.576)
     "chat70b": 1_470_800_000,     # profiles/attention_persist_chat70b_ncu.md
     "prefix_fp8": 157_300_000,    # profiles/attention_tma_e4m3_prefix_fp8_ncu.md
