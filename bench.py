@@ -16,7 +16,8 @@ and the headline record carries both figures) and timed by its own pair of CUDA 
 stream; the step time is the MEDIAN of the K. The same K steps run back to back without
 flushes are reported beside it. Prints ONE JSON line on rank 0: the headline workload (llama8b) at the
 top level and, at one GPU, the other graded configurations under ``also``, each with its own clock
-record and a parity flag from the oracle pass that is also its CPU baseline. With N > 1 (torchrun) every
+record and a parity flag from the oracle pass that is also its CPU baseline (a batch with a shared
+prefix also carries the same step through the shared-prefix cascade, under ``cascade``). With N > 1 (torchrun) every
 rank runs its own independent batch (sequences shard with no collective), the step time is the max over
 ranks and the value sums the ranks' bytes.
 """
@@ -235,7 +236,7 @@ def read_ceiling(dev, stream, reps=8):
     return READ_PROBE_BYTES / (best * 1e-3) / 1e9
 
 
-def run_workload(name, args, ctx, headline):
+def run_workload(name, args, ctx, headline, mode=None):
     """Times one workload on this rank's GPU; returns the rank-0 record (None on other ranks)."""
     import torch
     import torch.distributed as dist
@@ -245,7 +246,7 @@ def run_workload(name, args, ctx, headline):
     world, rank, dev, stream = ctx["world"], ctx["rank"], ctx["dev"], ctx["stream"]
     w = make(name, rank, args.batch)
     chunk = DEFAULT_CHUNK[w.name] if args.chunk is None or not headline else args.chunk
-    mode = args.mode if headline else "decode"
+    mode = mode or (args.mode if headline else "decode")
     if args.chunk is None and mode == "verify" and chunk:
         chunk *= 2   # a multi-query unit costs more to start than a decode unit: larger chunks (4096 for longctx)
     to16 = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
@@ -526,7 +527,7 @@ def run_workload(name, args, ctx, headline):
                       "d2h_bytes_per_step": e2e[2],
                       "mode": e2e[3], "staged_ms_per_step": e2e[4][0], "in_place_ms_per_step": e2e[4][1],
                       "all_in_place_ms_per_step": e2e[4][2]}
-    if world == 1 and not args.no_cpu_baseline and mode == "decode":
+    if world == 1 and not args.no_cpu_baseline and mode in ("decode", "cascade"):  # (the cascade's result is the same)
         # The oracle as it stands, timed on the host cores on this very batch; its result is also what
         # the GPU output of the timed steps is checked against, element by element (no throughput is
         # reported for a workload that fails).
@@ -584,6 +585,12 @@ def run_gpu(args):
         for name in names:
             if name != args.workload:
                 also[name] = run_workload(name, args, ctx, headline=False)
+                if name in PREFIX_TOKENS and rank == 0:
+                    # a batch with a shared prefix: the same step through paged_prefix_decode_attention (the
+                    # prefix read once for the whole batch) beside the plain decode step
+                    c = run_workload(name, args, ctx, headline=False, mode="cascade")
+                    also[name]["cascade"] = {k: c[k] for k in ("ms_per_step", "attention_ms", "back_to_back_ms_per_step",
+                                                               "value", "clocks", "parity", "gpu_launches") if k in c}
     if rank == 0:
         if head.get("parity") and not head["parity"]["ok"]:
             raise RuntimeError(f"parity check failed on {args.workload}: {head['parity']}")
