@@ -380,6 +380,24 @@ def run_workload(name, args, ctx, headline, mode=None):
     if int(status.item()) != 0:
         raise RuntimeError(f"device status {int(status.item())}: {pda.status_string(int(status.item()))}")
 
+    # ---- the flushed step once more without per-step events: K x (flush + step) minus K x flush, one event
+    # pair each. An event pair resolves about 2 us and puts a gap before the launch it brackets; the
+    # difference of the two totals does neither (it is printed beside the median, not instead of it).
+    ms_by_diff = None
+    if args.flush != "none":
+        def total(with_step):
+            a, b = new_event(), new_event()
+            barrier()
+            a.record(stream)
+            for i in range(K):
+                flush(i)
+                if with_step:
+                    step()
+            b.record(stream)
+            barrier()
+            return a.elapsed_time(b) / K
+        ms_by_diff = total(True) - total(False)
+
     # ---- headline only: the other flush, for the record (median of K, same event placement) -------------
     ms_other_flush = None
     if headline and args.flush != "none":
@@ -516,6 +534,8 @@ def run_workload(name, args, ctx, headline, mode=None):
         "clocks": sampler.summary(),
         "dtype": "bf16" if w.kv_dtype == "bf16" else "e4m3",
     }
+    if ms_by_diff is not None:
+        rec["ms_per_step_by_difference"] = ms_by_diff
     if ms_other_flush:
         rec["ms_per_step_after_" + ms_other_flush[0] + "_flush"] = ms_other_flush[1]
     if ms_graph > 0:
