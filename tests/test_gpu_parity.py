@@ -115,6 +115,9 @@ RAGGED = [
     ([3, 100, 513], 8, 8, 128),          # G = 1
     ([7, 64, 200], 6, 3, 64),            # G = 2
     ([9, 130], 24, 2, 96),               # G = 12, head_dim 96: generic kernel only
+    ([4, 33, 260, 1030], 12, 4, 128),    # G = 3
+    ([4, 33, 260, 1030], 20, 4, 128),    # G = 5
+    ([6, 70, 515], 28, 4, 128),          # G = 7
 ]
 
 

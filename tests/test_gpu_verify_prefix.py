@@ -405,3 +405,32 @@ def test_verify_fp8_persistent_kernel_edge_cases(oracle, T):
         torch.cuda.synchronize()
         assert torch.equal(res.view(torch.int16), out.view(torch.int16))
     assert int(dw.status.item()) == 0
+
+
+@pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
+@pytest.mark.parametrize("shape", [(6, 2), (20, 4), (28, 4), (12, 1)], ids=lambda s: f"Hq{s[0]}kv{s[1]}")
+def test_verify_group_sizes_that_are_not_powers_of_two(oracle, shape, kv_dtype):
+    """Query row r of a (sequence, kv head) unit is (draft token r / G, head r % G): G = 3, 5, 7 and 12, with
+    row counts that end inside a warp's 32 rows (T = 5: 15, 25, 35, 60 rows), fill one block exactly or not
+    (T = 16: 48, 80, 112, 192 rows) and need two blocks. Enough sequences that the persistent kernels carry
+    several units per CTA; the one-unit and the mma.sync kernels on the same inputs."""
+    Hq, Hkv = shape
+    rng = np.random.default_rng(500 + Hq)
+    B = -(-330 // Hkv)                      # more than 2 x 148 units
+    lens = np.maximum(rng.integers(1, 500, size=B), 16)
+    lens[:3] = [16, 64, 65]
+    w = W.make_workload("odd_group", lens, Hq, Hkv, 128, kv_dtype=kv_dtype, seed=501 + Hq)
+    for T in (5, 16):
+        q, kn, vn = verify_inputs(w, T, 502 + T)
+        k, v = w.k_cache.copy(), w.v_cache.copy()
+        dw = DeviceWorkload(w)
+        if kv_dtype == "bf16":
+            oracle.kv_append_tokens(kn, vn, k, v, w.block_table, w.seq_lens)
+            pda.kv_append_tokens(bf16_tensor(kn), bf16_tensor(vn), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens)
+        ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale, w.k_scale, w.v_scale)
+        for flags in (0, pda.PDA_FLAG_MQ_ONE_UNIT, pda.PDA_FLAG_MQ_MMA_SYNC):
+            out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                             float(w.scale), k_scale=dw.k_scale, v_scale=dw.v_scale, flags=flags,
+                                             status=dw.status)
+            assert_close(bf16_to_f64(out), ref, kv_dtype, what=f"G={Hq // Hkv} T={T} {kv_dtype} flags {flags}")
+    assert int(dw.status.item()) == 0
