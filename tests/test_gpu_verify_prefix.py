@@ -434,3 +434,28 @@ def test_verify_group_sizes_that_are_not_powers_of_two(oracle, shape, kv_dtype):
                                              status=dw.status)
             assert_close(bf16_to_f64(out), ref, kv_dtype, what=f"G={Hq // Hkv} T={T} {kv_dtype} flags {flags}")
     assert int(dw.status.item()) == 0
+
+
+@pytest.mark.parametrize("flags", MQ)
+def test_verify_sequences_shorter_than_the_block(oracle, flags):
+    """A sequence with fewer tokens than the block has query tokens (position L - n + i < 0 for the first
+    n - L of them): those rows attend nothing and are zero, the others follow the rule; an empty sequence
+    gives zero rows. Among them enough ordinary sequences for several units per CTA."""
+    T = 16
+    lens = [0, 1, 5, 15, 16, 17, 0, 3] + [20 + 7 * i for i in range(40)]
+    w = W.make_workload("short", lens, 32, 8, 128, seed=610)
+    q, _, _ = verify_inputs(w, T, 611)
+    k, v = w.k_cache.copy(), w.v_cache.copy()
+    oracle.kv_append(w.k_new, w.v_new, k, v, w.block_table, w.seq_lens)   # (the workload's last token)
+    ref, _ = oracle.paged_verify_attention(q, k, v, w.block_table, w.seq_lens, w.scale)
+    for b, L in enumerate(lens[:8]):
+        assert (ref[b, :max(T - L, 0)] == 0).all() and (L == 0 or np.abs(ref[b, T - 1]).max() > 0)
+    dw = DeviceWorkload(w)
+    dw.append()
+    out = pda.paged_verify_attention(bf16_tensor(q), dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens,
+                                     float(w.scale), flags=flags, status=dw.status)
+    got = bf16_to_f64(out)
+    assert_close(got, ref, what="verify with sequences shorter than the block")
+    for b, L in enumerate(lens[:8]):
+        assert (got[b, :max(T - L, 0)] == 0).all()
+    assert int(dw.status.item()) == 0
