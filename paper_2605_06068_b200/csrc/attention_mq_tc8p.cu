@@ -121,11 +121,24 @@ attention_mq_tc8p_kernel(const __grid_constant__ CUtensorMap k_map,
   // lengths, and the order of the sequences by length (longest first, ties by index): order_sh[rank] = j
   for (int j = tid; j < p.batch; j += kEThreads) lens_sh[j] = max(p.seq_lens[j], 0);
   __syncthreads();
-  for (int j = tid; j < p.batch; j += kEThreads) {
-    const int Lj = lens_sh[j];
-    int rank = 0;
-    for (int i = 0; i < p.batch; ++i) rank += (lens_sh[i] > Lj) || (lens_sh[i] == Lj && i < j);
-    order_sh[rank] = static_cast<uint16_t>(j);
+  {
+    // (one key per sequence, (length << 10) | (1023 - index): distinct and larger for the sequence that
+    // comes first; a rank is the number of larger keys, counted four keys to a load. The keys lie in the
+    // ring, which no copy has been sent to yet. Lengths from 2^21 on rank as equal.)
+    uint32_t* keys = reinterpret_cast<uint32_t*>(smem);
+    const int n_keys = (p.batch + 3) & ~3;
+    for (int j = tid; j < n_keys; j += kEThreads)
+      keys[j] = j < p.batch ? (static_cast<uint32_t>(min(lens_sh[j], (1 << 21) - 1)) << 10) | static_cast<uint32_t>(1023 - j) : 0u;
+    __syncthreads();
+    for (int j = tid; j < p.batch; j += kEThreads) {
+      const uint32_t kj = keys[j];
+      int rank = 0;
+      for (int i = 0; i < n_keys; i += 4) {
+        const uint4 k4 = *reinterpret_cast<const uint4*>(keys + i);
+        rank += (k4.x > kj) + (k4.y > kj) + (k4.z > kj) + (k4.w > kj);
+      }
+      order_sh[rank] = static_cast<uint16_t>(j);
+    }
   }
   tc_fence_before();
   __syncthreads();

@@ -147,10 +147,21 @@ attention_mq_tcp_kernel(const __grid_constant__ CUtensorMap k_map,
   for (int j = tid; j < p.batch; j += kPThreads) lens_sh[j] = max(p.seq_lens[j], 0);
   __syncthreads();
   if (p.batch <= kPSortBatch) {
+    // (one key per sequence, (length << 9) | (511 - index): distinct and larger for the sequence that comes
+    // first; a rank is the number of larger keys, counted four keys to a load. The keys lie in the ring,
+    // which no copy has been sent to yet. Lengths from 2^22 on rank as equal.)
+    uint32_t* keys = reinterpret_cast<uint32_t*>(smem);
+    const int n_keys = (p.batch + 3) & ~3;
+    for (int j = tid; j < n_keys; j += kPThreads)
+      keys[j] = j < p.batch ? (static_cast<uint32_t>(min(lens_sh[j], (1 << 22) - 1)) << 9) | static_cast<uint32_t>(511 - j) : 0u;
+    __syncthreads();
     if (tid < p.batch) {
-      const int Lj = lens_sh[tid];
+      const uint32_t kj = keys[tid];
       int rank = 0;
-      for (int i = 0; i < p.batch; ++i) rank += (lens_sh[i] > Lj) || (lens_sh[i] == Lj && i < tid);
+      for (int i = 0; i < n_keys; i += 4) {
+        const uint4 k4 = *reinterpret_cast<const uint4*>(keys + i);
+        rank += (k4.x > kj) + (k4.y > kj) + (k4.z > kj) + (k4.w > kj);
+      }
       order_sh[rank] = static_cast<uint16_t>(tid);
     }
   } else {

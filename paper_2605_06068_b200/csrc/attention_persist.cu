@@ -84,12 +84,24 @@ attention_persist_kernel(const __grid_constant__ CUtensorMap k_map,
     fence_proxy_async();
   }
   if (tid < 8) misc[tid] = 0;
-  for (int j = tid; j < B; j += kThreads) lens[j] = max(p.seq_lens[j], 0);
+  // (one key per sequence, (length << 8) | (255 - index): distinct and larger for the sequence that comes
+  // first; a rank is the number of larger keys, counted four keys to a load. The keys lie in the ring,
+  // which no copy has been sent to yet. Lengths from 2^23 on rank as equal.)
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem);
+  const int n_keys = (B + 3) & ~3;
+  for (int j = tid; j < n_keys; j += kThreads) {
+    const int Lj = j < B ? max(p.seq_lens[j], 0) : 0;
+    if (j < B) lens[j] = Lj;
+    keys[j] = j < B ? (static_cast<uint32_t>(min(Lj, (1 << 23) - 1)) << 8) | static_cast<uint32_t>(255 - j) : 0u;
+  }
   __syncthreads();
   for (int j = tid; j < B; j += kThreads) {
-    const int Lj = lens[j];
+    const uint32_t kj = keys[j];
     int rank = 0;
-    for (int i = 0; i < B; ++i) rank += (lens[i] > Lj) || (lens[i] == Lj && i < j);
+    for (int i = 0; i < n_keys; i += 4) {
+      const uint4 k4 = *reinterpret_cast<const uint4*>(keys + i);
+      rank += (k4.x > kj) + (k4.y > kj) + (k4.z > kj) + (k4.w > kj);
+    }
     order[rank] = j;
   }
   if (tid == 0) misc[0] = atomicAdd(&ws[0], 1);

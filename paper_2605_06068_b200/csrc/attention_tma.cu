@@ -76,14 +76,34 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
     // unsplit units differ in length by the spread of seq_lens: serve the longest first. The CTA
     // with blockIdx.z = r takes the r-th longest sequence (ties by index), so long units start
     // early and short ones fill the tail. (Split units are bounded by chunk_tokens already.)
-    int* lens = reinterpret_cast<int*>(smem);
-    for (int j = tid; j < p.batch; j += kWarps * 32) lens[j] = max(p.seq_lens[j], 0);
+    // One key per sequence, (length << 8) | (255 - index): distinct, and larger for the sequence that comes
+    // first. A sequence's rank is the number of larger keys, counted four keys to a shared-memory load
+    // (every CTA does this on its way to its first tile: with a compare on length and index per pair it
+    // cost a launch of 256 sequences 22 of 122 us). Lengths from 2^23 on rank as equal.
+    uint32_t* keys = reinterpret_cast<uint32_t*>(smem);
+    constexpr int kPerThread = (kMaxLptBatch + kWarps * 32 - 1) / (kWarps * 32);
+    const int n_keys = (p.batch + 3) & ~3;
+    int l_mine[kPerThread];
+#pragma unroll
+    for (int k = 0; k < kPerThread; ++k) {
+      const int j = tid + k * kWarps * 32;
+      l_mine[k] = j < p.batch ? max(p.seq_lens[j], 0) : 0;
+      if (j < n_keys)
+        keys[j] = j < p.batch ? (static_cast<uint32_t>(min(l_mine[k], (1 << 23) - 1)) << 8) | static_cast<uint32_t>(255 - j)
+                              : 0u;  // (padding: smaller than every key)
+    }
     __syncthreads();
-    for (int j = tid; j < p.batch; j += kWarps * 32) {
-      const int Lj = lens[j];
+#pragma unroll
+    for (int k = 0; k < kPerThread; ++k) {
+      const int j = tid + k * kWarps * 32;
+      if (j >= p.batch) break;
+      const uint32_t kj = keys[j];
       int rank = 0;
-      for (int i = 0; i < p.batch; ++i) rank += (lens[i] > Lj) || (lens[i] == Lj && i < j);
-      if (rank == static_cast<int>(blockIdx.z)) { cta_err[2] = j; cta_err[3] = Lj; }
+      for (int i = 0; i < n_keys; i += 4) {
+        const uint4 k4 = *reinterpret_cast<const uint4*>(keys + i);
+        rank += (k4.x > kj) + (k4.y > kj) + (k4.z > kj) + (k4.w > kj);
+      }
+      if (rank == static_cast<int>(blockIdx.z)) { cta_err[2] = j; cta_err[3] = l_mine[k]; }
     }
     __syncthreads();
     b = cta_err[2];
