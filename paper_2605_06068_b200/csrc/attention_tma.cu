@@ -29,6 +29,8 @@
 // Every wait on an mbarrier is bounded; on expiry the CTA reports
 // PDA_DEV_TIMEOUT, waits (bounded) for its copies in flight and zero-fills its
 // output. TMA copies never use multicast.
+#include <atomic>
+
 #include "common.cuh"
 #include "decode_tile.cuh"
 #include "tma_ptx.cuh"
@@ -59,7 +61,7 @@ struct Cfg {
 template <int D, bool kFp8, int kStages, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
 attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
-                     const __grid_constant__ CUtensorMap v_map, StepParams sp) {
+                     const __grid_constant__ CUtensorMap v_map, StepParams sp, int longest_first) {
   using C = Cfg<D, kFp8, kStages, kWarps>;
   const AttnParams& p = sp.a;
   extern __shared__ uint8_t smem_raw[];
@@ -72,38 +74,82 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
   const int c = blockIdx.x, g = blockIdx.y;
   int b = blockIdx.z;
   int L_ranked = -1;  // the unit's length when the ranking below has it at hand (saves a trip to memory)
-  if (p.chunk_tokens == 0 && p.batch <= kMaxLptBatch && p.batch > 1) {
+  if (longest_first) {  // (the host: unsplit, 2 .. kMaxLptBatch sequences, few units per resident CTA)
     // unsplit units differ in length by the spread of seq_lens: serve the longest first. The CTA
-    // with blockIdx.z = r takes the r-th longest sequence (ties by index), so long units start
-    // early and short ones fill the tail. (Split units are bounded by chunk_tokens already.)
-    // One key per sequence, (length << 8) | (255 - index): distinct, and larger for the sequence that comes
-    // first. A sequence's rank is the number of larger keys, counted four keys to a shared-memory load
-    // (every CTA does this on its way to its first tile: with a compare on length and index per pair it
-    // cost a launch of 256 sequences 22 of 122 us). Lengths from 2^23 on rank as equal.
-    uint32_t* keys = reinterpret_cast<uint32_t*>(smem);
-    constexpr int kPerThread = (kMaxLptBatch + kWarps * 32 - 1) / (kWarps * 32);
-    const int n_keys = (p.batch + 3) & ~3;
-    int l_mine[kPerThread];
+    // with blockIdx.z = r takes the sequence at place r of an order by decreasing length, so long units
+    // start early and short ones fill the tail. (Split units are bounded by chunk_tokens already. With more
+    // than about four units per resident CTA the order costs more than it gives: units of like length then
+    // run side by side and start side by side, and the HBM idles while they do. Measured on random lengths
+    // of 32..2048, bf16, one CTA per unit: 160 sequences 6.05 TB/s in this order, 6.33 as they come; 192:
+    // 6.24 and 6.53; 256: 6.50 and 6.62; at 128 sequences, 3.5 units per resident CTA, the order gives 6 %.)
+    // Every CTA does this on its way to its first tile, so it has to be cheap: counting, for every sequence,
+    // the sequences that come before it cost a 256-sequence launch 22 of 122 us (and 8-10 % from 160
+    // sequences up even four keys to a load). Instead: 64 buckets by length (longer first; the bucket
+    // width is the largest length / 64 rounded up to a power of two), by index inside a bucket. A warp
+    // handles 32 consecutive sequences at a time and finds a sequence's place among those of its bucket
+    // with a match; the counts per (32 sequences, bucket) are summed up by one warp. Every CTA computes the
+    // same order. 128 threads, up to 256 sequences: two per thread.
+    static_assert(kWarps == 4 && kMaxLptBatch == 256, "two sequences per thread, chunks of 32 by warp");
+    int* hist = reinterpret_cast<int*>(smem);   // [8 chunks][64 buckets]: sequences of the bucket in the chunk,
+                                                // then: in the chunks before it
+    int* offset = hist + 8 * 64;                // [64] sequences in the buckets above
+    int* wmax = offset + 64;                    // [4]
+    int l_mine[2];
+    int lmax = 0;
 #pragma unroll
-    for (int k = 0; k < kPerThread; ++k) {
-      const int j = tid + k * kWarps * 32;
+    for (int k = 0; k < 2; ++k) {
+      const int j = tid + 128 * k;
       l_mine[k] = j < p.batch ? max(p.seq_lens[j], 0) : 0;
-      if (j < n_keys)
-        keys[j] = j < p.batch ? (static_cast<uint32_t>(min(l_mine[k], (1 << 23) - 1)) << 8) | static_cast<uint32_t>(255 - j)
-                              : 0u;  // (padding: smaller than every key)
+      lmax = max(lmax, l_mine[k]);
+    }
+    for (int i = tid; i < 8 * 64; i += 128) hist[i] = 0;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) lmax = max(lmax, __shfl_xor_sync(0xffffffffu, lmax, off));
+    if (lane == 0) wmax[warp] = lmax;
+    __syncthreads();
+    lmax = max(max(wmax[0], wmax[1]), max(wmax[2], wmax[3]));
+    const int shift = max(32 - __clz(lmax) - 6, 0);  // lmax >> shift < 64
+    int bkt[2], ord[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int j = tid + 128 * k;
+      bkt[k] = j < p.batch ? (l_mine[k] >> shift) : 64 + lane;  // (no sequence: a bucket of its own, not counted)
+      const unsigned same = __match_any_sync(0xffffffffu, bkt[k]);
+      ord[k] = __popc(same & ((1u << lane) - 1u));
+      if (ord[k] == 0 && j < p.batch) hist[(warp + 4 * k) * 64 + bkt[k]] = __popc(same);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      int tot[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {  // buckets lane and lane + 32: counts -> counts in the chunks before
+        int run = 0;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const int x = hist[ch * 64 + lane + 32 * h];
+          hist[ch * 64 + lane + 32 * h] = run;
+          run += x;
+        }
+        tot[h] = run;
+      }
+      int s_lo = tot[0], s_hi = tot[1];  // -> sums over the buckets from this one up, within each half
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int y_lo = __shfl_down_sync(0xffffffffu, s_lo, off), y_hi = __shfl_down_sync(0xffffffffu, s_hi, off);
+        if (lane + off < 32) { s_lo += y_lo; s_hi += y_hi; }
+      }
+      const int all_hi = __shfl_sync(0xffffffffu, s_hi, 0);
+      offset[lane + 32] = s_hi - tot[1];
+      offset[lane] = s_lo - tot[0] + all_hi;
     }
     __syncthreads();
 #pragma unroll
-    for (int k = 0; k < kPerThread; ++k) {
-      const int j = tid + k * kWarps * 32;
-      if (j >= p.batch) break;
-      const uint32_t kj = keys[j];
-      int rank = 0;
-      for (int i = 0; i < n_keys; i += 4) {
-        const uint4 k4 = *reinterpret_cast<const uint4*>(keys + i);
-        rank += (k4.x > kj) + (k4.y > kj) + (k4.z > kj) + (k4.w > kj);
+    for (int k = 0; k < 2; ++k) {
+      const int j = tid + 128 * k;
+      if (j < p.batch && offset[bkt[k]] + hist[(warp + 4 * k) * 64 + bkt[k]] + ord[k] == static_cast<int>(blockIdx.z)) {
+        cta_err[2] = j;
+        cta_err[3] = l_mine[k];
       }
-      if (rank == static_cast<int>(blockIdx.z)) { cta_err[2] = j; cta_err[3] = l_mine[k]; }
     }
     __syncthreads();
     b = cta_err[2];
@@ -443,7 +489,20 @@ cudaError_t launch(const StepParams& sp, cudaStream_t stream) {
   if (e != cudaSuccess) return e;
   const unsigned chunks = p.chunk_tokens > 0 ? static_cast<unsigned>(p.max_chunks - p.chunk_slot0) : 1u;
   dim3 grid(chunks, p.geom.num_kv_heads, p.batch);
-  kern<<<grid, kWarps * 32, C::kSmemBytes, stream>>>(k_map, v_map, sp);
+  int longest_first = 0;
+  if (p.chunk_tokens == 0 && p.batch > 1 && p.batch <= kMaxLptBatch) {
+    static std::atomic<int> resident_per_sm{0};  // of this instance of the kernel (the same on every device of a process)
+    int per_sm = resident_per_sm.load();
+    if (per_sm == 0) {
+      if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kWarps * 32, C::kSmemBytes)) != cudaSuccess) return e;
+      resident_per_sm.store(per_sm);
+    }
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    longest_first = static_cast<int64_t>(p.batch) * p.geom.num_kv_heads <= 4ll * sms * per_sm;
+  }
+  kern<<<grid, kWarps * 32, C::kSmemBytes, stream>>>(k_map, v_map, sp, longest_first);
   return cudaGetLastError();
 }
 
