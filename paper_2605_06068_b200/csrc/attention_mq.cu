@@ -217,10 +217,13 @@ attention_mq_kernel(const __grid_constant__ CUtensorMap k_map,
         for (int ks = 0; ks < C::kKSteps; ks += 2) {
           uint32_t r[4];
           ldsm_x4(kt + tile_off(kb_row, ks + kb_chk), r);  // r0: tok 0-7 chunk ks, r1: tok 8-15 chunk ks, r2/r3: chunk ks+1
-          mma16816<true>(s0, qf[ks], e4m3x2_to_f16x2(r[0]), e4m3x2_to_f16x2(r[0] >> 16));
-          mma16816<true>(s1, qf[ks], e4m3x2_to_f16x2(r[1]), e4m3x2_to_f16x2(r[1] >> 16));
-          mma16816<true>(s0, qf[ks + 1], e4m3x2_to_f16x2(r[2]), e4m3x2_to_f16x2(r[2] >> 16));
-          mma16816<true>(s1, qf[ks + 1], e4m3x2_to_f16x2(r[3]), e4m3x2_to_f16x2(r[3] >> 16));
+          uint32_t c[4][2];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) e4m3x4_to_f16x2x2(r[i], c[i][0], c[i][1]);
+          mma16816<true>(s0, qf[ks], c[0][0], c[0][1]);
+          mma16816<true>(s1, qf[ks], c[1][0], c[1][1]);
+          mma16816<true>(s0, qf[ks + 1], c[2][0], c[2][1]);
+          mma16816<true>(s1, qf[ks + 1], c[3][0], c[3][1]);
         }
       }
       const float sc = scale_log2 * ksc;
@@ -291,10 +294,13 @@ attention_mq_kernel(const __grid_constant__ CUtensorMap k_map,
 #pragma unroll
           for (int e = 0; e < 4; ++e) r[e] = __byte_perm(r[e], 0, 0x3120);
           // output tile 2j: columns n <-> d = 16j + 2n ; tile 2j+1: d = 16j + 2n + 1 (and likewise for chunk j+1)
-          mma16816<true>(o[2 * j], pa, e4m3x2_to_f16x2(r[0]) & keep0, e4m3x2_to_f16x2(r[1]) & keep1);
-          mma16816<true>(o[2 * j + 1], pa, e4m3x2_to_f16x2(r[0] >> 16) & keep0, e4m3x2_to_f16x2(r[1] >> 16) & keep1);
-          mma16816<true>(o[2 * j + 2], pa, e4m3x2_to_f16x2(r[2]) & keep0, e4m3x2_to_f16x2(r[3]) & keep1);
-          mma16816<true>(o[2 * j + 3], pa, e4m3x2_to_f16x2(r[2] >> 16) & keep0, e4m3x2_to_f16x2(r[3] >> 16) & keep1);
+          uint32_t c[4][2];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) e4m3x4_to_f16x2x2(r[i], c[i][0], c[i][1]);
+          mma16816<true>(o[2 * j], pa, c[0][0] & keep0, c[1][0] & keep1);
+          mma16816<true>(o[2 * j + 1], pa, c[0][1] & keep0, c[1][1] & keep1);
+          mma16816<true>(o[2 * j + 2], pa, c[2][0] & keep0, c[3][0] & keep1);
+          mma16816<true>(o[2 * j + 3], pa, c[2][1] & keep0, c[3][1] & keep1);
         }
       }
 

@@ -87,11 +87,11 @@ __device__ __forceinline__ void decode_tile(uint32_t kt, uint32_t vt, int n_vali
       for (int ks = 0; ks < kKSteps; ks += 2) {
         uint32_t r[4], a[4];
         ldsm_x4(kt + tile_off(k_row, ks + k_chk), r);   // r0,r1: chunk ks rows 0-7 / 8-15; r2,r3: chunk ks+1
-        a[0] = e4m3x2_to_f16x2(r[0]); a[2] = e4m3x2_to_f16x2(r[0] >> 16);
-        a[1] = e4m3x2_to_f16x2(r[1]); a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+        e4m3x4_to_f16x2x2(r[0], a[0], a[2]);
+        e4m3x4_to_f16x2x2(r[1], a[1], a[3]);
         mma16816<true>(sa, a, qf[ks][0], qf[ks][1]);
-        a[0] = e4m3x2_to_f16x2(r[2]); a[2] = e4m3x2_to_f16x2(r[2] >> 16);
-        a[1] = e4m3x2_to_f16x2(r[3]); a[3] = e4m3x2_to_f16x2(r[3] >> 16);
+        e4m3x4_to_f16x2x2(r[2], a[0], a[2]);
+        e4m3x4_to_f16x2x2(r[3], a[1], a[3]);
         mma16816<true>(sb, a, qf[ks + 1][0], qf[ks + 1][1]);
       }
     }
@@ -139,11 +139,11 @@ __device__ __forceinline__ void decode_tile(uint32_t kt, uint32_t vt, int n_vali
         // with dA = 16*chunk + 2gid: regroup to (V[2tq][d], V[2tq+1][d]) pairs for d = dA, dA+1
 #pragma unroll
         for (int i = 0; i < 4; ++i) r[i] = __byte_perm(r[i], 0, 0x3120);
-        a[0] = e4m3x2_to_f16x2(r[0]); a[1] = e4m3x2_to_f16x2(r[0] >> 16);
-        a[2] = e4m3x2_to_f16x2(r[1]); a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+        e4m3x4_to_f16x2x2(r[0], a[0], a[1]);
+        e4m3x4_to_f16x2x2(r[1], a[2], a[3]);
         mma16816<true>(o[mt], a, pb0, pb1);
-        a[0] = e4m3x2_to_f16x2(r[2]); a[1] = e4m3x2_to_f16x2(r[2] >> 16);
-        a[2] = e4m3x2_to_f16x2(r[3]); a[3] = e4m3x2_to_f16x2(r[3] >> 16);
+        e4m3x4_to_f16x2x2(r[2], a[0], a[1]);
+        e4m3x4_to_f16x2x2(r[3], a[2], a[3]);
         mma16816<true>(o[mt + 1], a, pb0, pb1);
       }
     }

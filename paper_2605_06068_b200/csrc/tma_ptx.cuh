@@ -148,6 +148,12 @@ __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
 }
 
 
+// four e4m3 bytes -> two f16x2 (bytes 0, 1 and bytes 2, 3), the halves of x taken as they lie
+__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t x, uint32_t& lo, uint32_t& hi) {
+  asm("{\n\t.reg .b16 t0, t1;\n\tmov.b32 {t0, t1}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, t0;\n\tcvt.rn.f16x2.e4m3x2 %1, t1;\n\t}"
+      : "=r"(lo), "=r"(hi) : "r"(x));
+}
+
 // Byte offset of 16-byte chunk `chunk` of row `r` inside a tile stored as
 // sub-tiles of [16 rows][128 B] with the 128-byte TMA swizzle.
 __device__ __forceinline__ uint32_t tile_off(int r, int chunk) {
