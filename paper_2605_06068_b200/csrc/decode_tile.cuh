@@ -119,9 +119,13 @@ __device__ __forceinline__ void decode_tile(uint32_t kt, uint32_t vt, int n_vali
     const uint32_t pb1 = movmatrix_trans(pack2<kFp8>(p2 * vsc, p3 * vsc));   // tokens 8-15
 
     // ---- O^T = O^T * alpha + V^T . P^T
+    // (after the first tiles of a unit the running maxima seldom move: alpha is exactly 1 then, and the
+    // 4 D / 16 multiplications are skipped when it is for the whole warp)
+    if (__any_sync(0xffffffffu, (al0 != 1.f) | (al1 != 1.f))) {
 #pragma unroll
-    for (int mt = 0; mt < kKSteps; ++mt) {
-      o[mt][0] *= al0; o[mt][1] *= al1; o[mt][2] *= al0; o[mt][3] *= al1;
+      for (int mt = 0; mt < kKSteps; ++mt) {
+        o[mt][0] *= al0; o[mt][1] *= al1; o[mt][2] *= al0; o[mt][3] *= al1;
+      }
     }
     if (!kFp8) {
 #pragma unroll
