@@ -56,7 +56,7 @@ NCU_TRAFFIC_BYTES = {
     "llama8b": 620_500_000,       # profiles/attention_tma_llama8b_ncu.md
     "longctx": 2_707_000_000,     # profiles/attention_tma_split_fused_longctx_ncu.md (2 of 8 sequences captured, x 4.576)
     "chat70b": 1_470_800_000,     # profiles/attention_persist_chat70b_ncu.md
-    "prefix_fp8": 157_300_000,    # profiles/attention_tma_e4m3_prefix_fp8_ncu.md
+    "prefix_fp8": 157_800_000,    # profiles/attention_tma_e4m3_prefix_fp8_ncu.md
 }
 TOL = {"bf16": (5e-3, 1e-2), "e4m3": (2e-2, 2e-2)}
 
