@@ -667,3 +667,25 @@ def test_fp8_block_append_bit_exact_and_verified(oracle, shape):
                                      k_scale=dks, v_scale=dvs, status=status)
     assert_close(bf16_to_f64(out), ref, "e4m3", what="verify after fp8 block appends")
     assert int(status.item()) == 0
+
+
+@pytest.mark.parametrize("kv_dtype", ["bf16", "e4m3"])
+@pytest.mark.parametrize("B", [2, 31, 33, 128, 129, 200, 256, 257])
+def test_longest_first_order_visits_every_sequence_once(oracle, B, kv_dtype):
+    """Unsplit launches of up to 256 sequences serve the sequences by decreasing length: 64 length buckets,
+    by index inside a bucket, every CTA computing the same order. Batches on either side of a warp's 32
+    sequences and of the 128 threads, with many equal lengths, empty sequences, and one sequence far longer
+    than the rest (which sets the bucket width): every row must be right, i.e. every sequence was taken by
+    exactly one CTA per kv head. 257 sequences: no ordering."""
+    rng = np.random.default_rng(900 + B)
+    lens = rng.integers(0, 40, size=B)
+    lens[rng.integers(0, B, size=max(B // 8, 1))] = 17          # ties
+    lens[rng.integers(0, B)] = 2100                             # one long sequence
+    w = W.make_workload("order", lens, 8, 2, 128, kv_dtype=kv_dtype, seed=901 + B)
+    dw = DeviceWorkload(w)
+    if kv_dtype == "bf16":
+        dw.append()
+    ref = oracle_out(oracle, w)
+    for rep in range(2):
+        assert_close(bf16_to_f64(dw.attend()), ref, kv_dtype, what=f"B={B} {kv_dtype} launch {rep}")
+    assert status_of(dw) == 0
