@@ -219,9 +219,8 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
 
   const uint32_t leader = elect_one();
   const uint64_t pol = l2_policy_evict_first();
-  auto issue = [&](int kk, int page_raw) {  // whole warp, converged; the elected lane issues
+  auto issue = [&](int s, int page_raw) {  // into stage s; whole warp, converged; the elected lane issues
     const int page = max(page_raw, 0);
-    const int s = kk % kStages;
     const uint32_t bar = bar0 + 8 * s;
     const uint32_t dst = ring + s * C::kStageBytes;
     mbar_expect_tx_if(leader, bar, C::kStageBytes);
@@ -269,12 +268,13 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
 
   bool timed_out = false;
   int kk = 0;
-  for (; kk < n_mine; ++kk) {
-    const int s = kk % kStages;
+  int s = 0;           // kk % kStages and the parity of kk / kStages, kept by counting (the kernel's
+  uint32_t phase = 0;  // instructions are what bounds it on e4m3 caches whose pages are shared)
+  int tok0 = (page0 + warp) * kPageSize;
+  for (; kk < n_mine; ++kk, tok0 += kWarps * kPageSize) {
     const uint32_t bar = bar0 + 8 * s;
-    if (!mbar_wait_bounded(bar, (kk / kStages) & 1)) { timed_out = true; break; }
+    if (!mbar_wait_bounded(bar, phase)) { timed_out = true; break; }
     const uint32_t kt = ring + s * C::kStageBytes, vt = kt + C::kTileBytes;
-    const int tok0 = (page0 + warp + kk * kWarps) * kPageSize;
     const int n_valid = min(kPageSize, t1 - tok0);  // rows [n_skip, n_valid) of the tile are attended
     const int n_skip = max(lo - tok0, 0);           // > 0 only in the unit's first tile
     float ksc = 1.f, vsc = 1.f;
@@ -317,8 +317,9 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap k_map,
       const int page = __shfl_sync(0xffffffffu, in_a ? pgA : pgB, kn & 31);
       if (page < 0) bad_page = true;
       fence_proxy_async();
-      issue(kn, page);
+      issue(s, page);  // (kn % kStages == kk % kStages)
     }
+    if (++s == kStages) { s = 0; phase ^= 1u; }
   }
 
   if (timed_out) {
