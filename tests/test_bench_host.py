@@ -36,3 +36,14 @@ def test_traffic_table_covers_the_workloads_of_the_default_line():
     for name in ["llama8b"] + bench.DEFAULT_ALSO:
         assert bench.NCU_TRAFFIC_BYTES.get(name), name
         assert name in bench.DEFAULT_CHUNK
+
+
+def test_prefix_chunk_rule():
+    """The cascade's default prefix chunk: at most one prefix CTA per SM, at least 1024 tokens, a power of two."""
+    class Shape:
+        def __init__(self, batch, hq, hkv):
+            self.batch, self.num_q_heads, self.num_kv_heads = batch, hq, hkv
+    assert bench.prefix_chunk_tokens(Shape(20, 32, 8), 32768) == 2048      # 8 units a chunk: 16 chunks, 128 CTAs
+    assert bench.prefix_chunk_tokens(Shape(128, 32, 8), 2048) == 1024      # 32 units a chunk: 4 chunks would be 512 tokens
+    assert bench.prefix_chunk_tokens(Shape(1, 8, 8), 100) == 1024
+    assert bench.prefix_chunk_tokens(Shape(4096, 64, 8), 1 << 20) == 1 << 20  # more units a chunk than SMs: one chunk
