@@ -262,7 +262,10 @@ int paged_verify_attention(const void* q, const void* k_cache, const void* v_cac
  *   block_table    rows must agree on their first prefix_tokens/page_size entries
  *                  (row 0's are used); prefix_tokens is a multiple of page_size and
  *                  <= every seq_lens[b]
- *   prefix_chunk_tokens  split of the prefix for parallelism (multiple of page_size)
+ *   prefix_chunk_tokens  split of the prefix for parallelism (multiple of page_size). The
+ *                  prefix launch has ceil(batch * group / 128) * num_kv_heads CTAs per chunk,
+ *                  each with a fixed cost of several microseconds: fastest with at most one
+ *                  CTA per SM and chunks of 1024 tokens or more
  *   chunk_tokens   (> 0) split of the suffixes
  *   part_o, part_lse  scratch [batch, num_q_heads, max_chunks, head_dim] / [.., max_chunks]
  *                  with max_chunks >= ceil(prefix_tokens/prefix_chunk_tokens)
